@@ -1,0 +1,370 @@
+#!/usr/bin/env python
+"""Benchmark of the draft + verify hot path (metric: draft+verify sequences/s).
+
+One step = one spec_draft (n heads, full product tree, prune to K) followed by one
+spec_verify over base_logits [B, K, n+1, V], on seeded synthetic inputs shaped like the
+BASELINE "Llama2-13B-shaped" configuration.  Prints ONE JSON line on rank 0.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--config NAME] [--impl ours|reference]
+
+N > 1 (under torchrun): sequences are independent, so every rank runs the full per-GPU
+batch with replicated weights and no data-path collective (weak scaling); the reported
+value is N * B / max-over-ranks step time.
+--impl reference times the CPU oracle (a deliberately plain program) on a bounded sample.
+"""
+from __future__ import annotations
+
+import argparse
+import dataclasses
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "draft+verify sequences/sec"
+UNIT = "sequences/s"
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return {"hbm_gbs": p["hbm_gbs"], "bf16_tflops": p["bf16_tflops"],
+                "bf16_tflops_sustained": p.get("bf16_tflops_sustained", p["bf16_tflops"]), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu_index = gpu_index
+        self.proc = None
+        self.lines = []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--id={self.gpu_index}", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for ln in self.lines:
+            parts = [x.strip() for x in ln.split(",")]
+            if len(parts) < 7:
+                continue
+            try:
+                sm.append(float(parts[0]))
+                mx.append(float(parts[1]))
+            except ValueError:
+                continue
+            for nm, val in zip(names, parts[3:7]):
+                if val.lower().startswith("active"):
+                    reasons.add(nm)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def oracle_weights(sw):
+    import oracle
+    from paper_2404_19124_b200 import synth
+    cfg = sw.cfg
+    return oracle.Weights(
+        V=cfg.V, d_base=cfg.d_base, d_inner=cfg.d_inner,
+        emb=[synth.bf16_bits(t) for t in sw.emb], proj=[synth.bf16_bits(t) for t in sw.proj],
+        ln_gamma=[t.detach().cpu().numpy() for t in sw.ln_gamma], ln_beta=[t.detach().cpu().numpy() for t in sw.ln_beta],
+        head=[synth.bf16_bits(t) for t in sw.head],
+        state_weight=sw.state_weight, emb_weight=sw.emb_weight, ln_eps=sw.ln_eps)
+
+
+def time_oracle(cfg, sw, seqs: int, repeats: int):
+    """Oracle draft + verify on the first `seqs` sequences of the workload; returns seconds per repeat."""
+    import numpy as np
+    import oracle
+    from paper_2404_19124_b200 import synth
+    ow = oracle_weights(sw)
+    ctx, tok = synth.make_draft_inputs(cfg, device="cpu", B=seqs)
+    ctx_bits, tok_np = synth.bf16_bits(ctx), tok.numpy()
+    cand0 = synth.random_cand_tok(cfg, B=seqs)
+    logits = synth.bf16_bits(synth.make_base_logits(cfg, cand0, B=seqs))
+    times = []
+    for _ in range(repeats):
+        t0 = time.perf_counter()
+        ct, _ = oracle.draft(ow, ctx_bits, tok_np, cfg.topk, cfg.K)
+        oracle.verify(ct, logits, oracle.BF16)
+        times.append(time.perf_counter() - t0)
+    return times, oracle.num_threads()
+
+
+def run_reference(args, cfg):
+    from paper_2404_19124_b200 import synth
+    seqs = 1
+    sw = synth.make_weights(cfg, device="cpu")
+    times, cores = time_oracle(cfg, sw, seqs, args.warmup + args.steps)
+    timed = times[args.warmup:]
+    sec = sum(timed) / len(timed)
+    val = seqs / sec
+    sample = f"{seqs} of {cfg.B} sequences of {cfg.name} per step (full tree + verify), plain C oracle, OpenMP"
+    out = {
+        "impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": sec * 1e3, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": cfg.name, "B": cfg.B, "K": cfg.K, "n_heads": cfg.n, "topk": list(cfg.topk),
+                   "V": cfg.V, "d_base": cfg.d_base, "d_inner": cfg.d_inner},
+        "cpu_baseline": {"value": val, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(out), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=20)
+    ap.add_argument("--config", default="llama2-13b")
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+
+    from paper_2404_19124_b200 import synth
+    cfg = synth.CONFIGS[args.config]
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+
+    if args.impl == "reference":
+        if rank == 0:
+            if args.steps == 200 and args.warmup == 20:      # defaults are sized for the GPU arm
+                args.steps, args.warmup = 3, 1
+            run_reference(args, cfg)
+        return
+
+    import torch
+    from paper_2404_19124_b200 import binding as B
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the draft/verify path has no CPU fallback")
+    torch.cuda.set_device(local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    if args.warmup < 3:
+        args.warmup = 3
+    peaks = load_peaks()
+    dev = f"cuda:{local_rank}"
+
+    # ---------------------------------------------------------------- inputs, resident in HBM
+    sw = synth.make_weights(cfg, device=dev)
+    h = B.spec_create(sw)
+    ctx, tok = synth.make_draft_inputs(cfg, device=dev)
+    n, K, Bn, V = cfg.n, cfg.K, cfg.B, cfg.V
+    ws = torch.empty(B.spec_draft_workspace_bytes(h, Bn, cfg.topk, K), dtype=torch.uint8, device=dev)
+    cand = torch.empty((Bn, K, n), dtype=torch.int32, device=dev)
+    logp = torch.empty((Bn, K), dtype=torch.float32, device=dev)
+    B.spec_draft(h, ctx, tok, cfg.topk, K, cand_tok=cand, cand_logp=logp, workspace=ws)
+    assert B.spec_poll_error(ws) == 0
+    # base-model logits: rotate over several distinct buffers so verify never re-reads a buffer that
+    # could still sit in the 126 MB L2; matches are planted at the tokens the draft proposes
+    logits_bytes = Bn * K * (n + 1) * V * 2
+    n_rot = max(2, min(8, (512 << 20) // logits_bytes + 1))
+    rot = [synth.make_base_logits(dataclasses.replace(cfg, seed=cfg.seed + 100 * i), cand, device=dev)
+           for i in range(n_rot)]
+    vws = torch.empty(B.spec_verify_workspace_bytes(Bn, K, n, V, B.SPEC_BF16), dtype=torch.uint8, device=dev)
+    acc = torch.empty(Bn, dtype=torch.int32, device=dev)
+    best = torch.empty(Bn, dtype=torch.int32, device=dev)
+    nxt = torch.empty(Bn, dtype=torch.int32, device=dev)
+    stream = torch.cuda.current_stream()
+
+    def step(i):
+        B.spec_draft(h, ctx, tok, cfg.topk, K, cand_tok=cand, cand_logp=logp, workspace=ws)
+        B.spec_verify(cand, rot[i % n_rot], accept_len=acc, best_cand=best, next_tok=nxt, workspace=vws)
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def max_over_ranks(x: float) -> float:
+        if dist is None:
+            return x
+        t = torch.tensor([x], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        return float(t.item())
+
+    # ---------------------------------------------------------------- device-resident timing
+    for i in range(args.warmup):
+        step(i)
+    barrier()
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
+        time.sleep(0.25)
+    barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for i in range(args.steps):
+        step(i)
+    e1.record(stream)
+    barrier()
+    ms_step = max_over_ranks(e0.elapsed_time(e1) / args.steps)
+    clocks = sampler.stop() if rank == 0 else None
+    assert B.spec_poll_error(ws) == 0
+    tau = float(acc.float().mean().item()) + 1.0
+
+    # ---------------------------------------------------------------- end to end from host buffers
+    pin = lambda t: t.cpu().pin_memory()
+    h_ctx, h_tok = pin(ctx), pin(tok)
+    h_rot = [pin(t) for t in rot[:2]]
+    d_logits = torch.empty_like(rot[0])
+    d_ctx, d_tok = torch.empty_like(ctx), torch.empty_like(tok)
+    h_cand = torch.empty(cand.shape, dtype=cand.dtype).pin_memory()
+    h_out = [torch.empty(Bn, dtype=torch.int32).pin_memory() for _ in range(3)]
+    h2d = h_ctx.numel() * 2 + h_tok.numel() * 4 + h_rot[0].numel() * 2
+    d2h = h_cand.numel() * 4 + 3 * Bn * 4
+
+    def e2e_step(i):
+        d_ctx.copy_(h_ctx, non_blocking=True)
+        d_tok.copy_(h_tok, non_blocking=True)
+        d_logits.copy_(h_rot[i % 2], non_blocking=True)
+        B.spec_draft(h, d_ctx, d_tok, cfg.topk, K, cand_tok=cand, cand_logp=logp, workspace=ws)
+        B.spec_verify(cand, d_logits, accept_len=acc, best_cand=best, next_tok=nxt, workspace=vws)
+        h_cand.copy_(cand, non_blocking=True)
+        for dst, src in zip(h_out, (acc, best, nxt)):
+            dst.copy_(src, non_blocking=True)
+        stream.synchronize()      # the caller needs the accepted tokens before the next step
+
+    e2e_steps = max(3, min(args.steps, 50))
+    for i in range(3):
+        e2e_step(i)
+    barrier()
+    t0 = time.perf_counter()
+    for i in range(e2e_steps):
+        e2e_step(i)
+    torch.cuda.synchronize()
+    e2e_ms = max_over_ranks((time.perf_counter() - t0) * 1e3 / e2e_steps)
+
+    # ---------------------------------------------------------------- per-kernel times (CUDA events)
+    B.spec_set_option(h, B.SPEC_OPT_PROFILE, 1)
+    prof_steps = max(3, min(args.steps, 50))
+    sums = None
+    for i in range(prof_steps):
+        step(i)
+        ms = B.spec_profile_read(h)
+        sums = ms if sums is None else [a + b for a, b in zip(sums, ms)]
+    kern_ms = [s / prof_steps for s in sums]
+    B.spec_set_option(h, B.SPEC_OPT_PROFILE, 0)
+    # verify alone, rotating buffers
+    v0, v1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    for i in range(3):
+        B.spec_verify(cand, rot[i % n_rot], accept_len=acc, best_cand=best, next_tok=nxt, workspace=vws)
+    torch.cuda.synchronize()
+    v0.record(stream)
+    for i in range(prof_steps):
+        B.spec_verify(cand, rot[i % n_rot], accept_len=acc, best_cand=best, next_tok=nxt, workspace=vws)
+    v1.record(stream)
+    torch.cuda.synchronize()
+    verify_ms = v0.elapsed_time(v1) / prof_steps
+
+    if rank != 0:
+        if dist is not None:
+            dist.destroy_process_group()
+        return
+
+    names = []
+    for l in range(n):
+        names += [f"proj_gemm[{l}]", f"mix_ln_gelu[{l}]", f"head_gemm[{l}]", f"merge_expand[{l}]"]
+    names.append("prune")
+    kernels = {nm: round(ms * 1e3, 2) for nm, ms in zip(names, kern_ms)}      # microseconds
+    # dominant kernel: the vocabulary-head GEMM of the last (widest) level
+    rows_last = cfg.nodes(n - 1)
+    head_ms = kern_ms[4 * (n - 1) + 2]
+    flops = 2.0 * rows_last * cfg.d_inner * V
+    w_bytes = 2.0 * V * cfg.d_inner + 2.0 * rows_last * cfg.d_inner
+    ridge = peaks["bf16_tflops"] * 1e12 / (peaks["hbm_gbs"] * 1e9)
+    if rows_last >= ridge:
+        ach = flops / (head_ms * 1e-3) / 1e12
+        roof = {"kernel": f"gemm_tc_kernel (vocabulary head, level {n - 1}: {rows_last} x {cfg.d_inner} x {V})",
+                "bound": "tensor", "achieved": ach, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
+                "frac": ach / peaks["bf16_tflops"], "traffic": None, "peak_source": peaks["source"] + " burst",
+                "frac_of_sustained": ach / peaks["bf16_tflops_sustained"]}
+    else:
+        ach = w_bytes / (head_ms * 1e-3) / 1e9
+        roof = {"kernel": f"gemm_tc_kernel (vocabulary head, level {n - 1}: {rows_last} x {cfg.d_inner} x {V})",
+                "bound": "hbm", "achieved": ach, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                "frac": ach / peaks["hbm_gbs"], "traffic": None, "peak_source": peaks["source"]}
+    v_gbs = logits_bytes / (verify_ms * 1e-3) / 1e9
+    roof_verify = {"kernel": "verify_argmax_kernel + verify_accept_kernel", "bound": "hbm", "achieved": v_gbs,
+                   "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": v_gbs / peaks["hbm_gbs"], "traffic": None,
+                   "us": round(verify_ms * 1e3, 2), "bytes": logits_bytes}
+    # heads below the ridge are weight-bandwidth bound: report their HBM fraction too
+    head_hbm = {}
+    for l in range(n):
+        hb = 2.0 * V * cfg.d_inner + 2.0 * cfg.nodes(l) * cfg.d_inner
+        head_hbm[f"head_gemm[{l}]"] = {"rows": cfg.nodes(l),
+                                       "GB/s": round(hb / (kern_ms[4 * l + 2] * 1e-3) / 1e9, 1),
+                                       "TFLOP/s": round(2.0 * cfg.nodes(l) * cfg.d_inner * V / (kern_ms[4 * l + 2] * 1e-3) / 1e12, 1)}
+
+    cpu = None
+    if world == 1 and not args.no_cpu_baseline:
+        seqs = 1
+        sw_cpu = synth.SpecWeights(cfg, *[[t.cpu() for t in lst] for lst in (sw.emb, sw.proj, sw.ln_gamma, sw.ln_beta, sw.head)],
+                                   sw.state_weight, sw.emb_weight, sw.ln_eps)
+        times, cores = time_oracle(cfg, sw_cpu, seqs, 2)
+        cpu = {"value": seqs / min(times), "unit": UNIT, "cores": cores, "kind": "oracle",
+               "sample": f"{seqs} of {Bn} sequences of {cfg.name} (full draft tree + verify), best of 2 runs, "
+                         f"{min(times):.2f} s"}
+
+    launches_per_step = 4 * n + 1 + 2
+    out = {
+        "metric": METRIC, "value": world * Bn / (ms_step * 1e-3), "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": cfg.name, "B": Bn, "K": K, "n_heads": n, "topk": list(cfg.topk), "V": V,
+                   "d_base": cfg.d_base, "d_inner": cfg.d_inner, "logits_dtype": "bf16",
+                   "l2": f"weights 1.7 GB+ per step exceed L2; verify rotates over {n_rot} distinct logits buffers",
+                   "parallelism": f"replicas x{world}, sequences independent, no collective"},
+        "roofline": roof, "roofline_verify": roof_verify, "head_gemms": head_hbm, "kernel_us": kernels,
+        "cpu_baseline": cpu,
+        "e2e": {"value": world * Bn / (e2e_ms * 1e-3), "unit": UNIT, "ms_per_step": e2e_ms,
+                "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
+        "gpu_launches": launches_per_step * args.steps,
+        "clocks": clocks, "synthetic_tokens_per_step": tau,
+    }
+    print(json.dumps(out), flush=True)
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -1,0 +1,161 @@
+/*
+ * spec_b200 - C ABI of the B200 (sm_100a) draft-tree generation and greedy verification
+ * library for the combined token/embedding speculator of arXiv 2404.19124.
+ *
+ * Conventions
+ *   - plain C, no exceptions cross the boundary; every call returns a SPEC_* status.
+ *   - "dev" pointers are CUDA device pointers, "host" pointers are ordinary host memory.
+ *   - the library never allocates or frees device memory: inputs, outputs, weights and
+ *     workspaces are owned by the caller and must stay valid until the work queued on
+ *     the stream has finished.
+ *   - spec_draft / spec_verify only enqueue work on `cuda_stream` (a cudaStream_t passed
+ *     as void*; NULL = default stream) and never synchronise.
+ *   - errors found on the host (bad pointers, shapes, workspace too small) are returned
+ *     at once and nothing is enqueued.  Errors found on the device (token id outside
+ *     [0, V), a bounded wait that ran out) are recorded in an error word at the start of
+ *     the workspace and reported by spec_poll_error; kernels never trap.
+ */
+#ifndef SPEC_B200_H_
+#define SPEC_B200_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define SPEC_MAX_HEADS 8     /* stages of the speculator (the paper uses 3, 5 and 7)         */
+#define SPEC_MAX_TOPK 8      /* branching factor of one head                                  */
+#define SPEC_MAX_LEAVES 4096 /* product of the branching factors, per sequence                */
+
+enum spec_status {
+    SPEC_OK = 0,
+    SPEC_ERR_INVALID_ARG = 1, /* null pointer, non-positive size, unknown dtype / option      */
+    SPEC_ERR_SHAPE = 2,       /* K > leaves, topk > SPEC_MAX_TOPK, widths not multiples of 8  */
+    SPEC_ERR_WORKSPACE = 3,   /* workspace missing, misaligned (256 B) or too small           */
+    SPEC_ERR_CUDA = 4,        /* a CUDA runtime/driver call failed: see spec_last_cuda_error  */
+    SPEC_ERR_TOKEN_RANGE = 5, /* device: a token id was outside [0, V) (its embedding is
+                                 treated as zero and the call runs to completion)             */
+    SPEC_ERR_TIMEOUT = 6,     /* device: a bounded wait inside a kernel ran out               */
+    SPEC_ERR_NO_DEVICE = 7    /* no CUDA device / not an sm_100 part                          */
+};
+
+enum spec_dtype { SPEC_BF16 = 0, SPEC_F32 = 1 };
+
+enum spec_option {
+    SPEC_OPT_GEMM_IMPL = 0,    /* 0 (default): tcgen05/TMEM tensor-core kernels; 1: slow CUDA-core
+                                  kernels kept for debugging the tensor-core path              */
+    SPEC_OPT_HEAD_BLOCK_N = 1, /* vocabulary columns per tile of the head GEMM; 0 = automatic  */
+    SPEC_OPT_PROJ_BLOCK_N = 2, /* output columns per tile of the state projection; 0 = auto    */
+    SPEC_OPT_PROFILE = 3       /* 1: spec_draft brackets each of its kernels with CUDA events on
+                                  the caller's stream (read them with spec_profile_read); costs a
+                                  few microseconds per call, off by default                    */
+};
+
+typedef struct spec_handle_s *spec_handle_t;
+
+/* Speculator parameters (Sec. 3.1: every stage has its own embedding table, state
+ * projection, LayerNorm and vocabulary output matrix; nothing is tied).  All pointers are
+ * dev, row-major, 16-byte aligned, read-only, caller-owned. */
+typedef struct {
+    int32_t n_heads, V, d_base, d_inner;   /* d_base % 8 == 0, d_inner % 8 == 0              */
+    const void *emb[SPEC_MAX_HEADS];       /* bf16 [V, d_inner]                               */
+    const void *proj[SPEC_MAX_HEADS];      /* bf16 [d_inner, d_in]; d_in = d_base for head 0,
+                                              d_inner for the others                          */
+    const float *ln_gamma[SPEC_MAX_HEADS]; /* fp32 [d_inner]                                  */
+    const float *ln_beta[SPEC_MAX_HEADS];  /* fp32 [d_inner]                                  */
+    const void *head[SPEC_MAX_HEADS];      /* bf16 [V, d_inner]                               */
+    float state_weight;                    /* a: weight of the projected state in the mix     */
+    float emb_weight;                      /* b: weight of the token embedding in the mix     */
+    float ln_eps;
+} spec_weights_t;
+
+/* Byte offsets into a draft workspace (for tests and debugging; N_l = B * prod_{j<l} topk[j]). */
+typedef struct {
+    uint64_t total_bytes;
+    uint64_t error_word;                  /* int32                                            */
+    uint64_t tok[SPEC_MAX_HEADS + 1];     /* int32 [N_l]: token of every node of level l>=1   */
+    uint64_t score[SPEC_MAX_HEADS + 1];   /* fp32  [N_l]: cumulative log-prob, level l>=1     */
+    uint64_t state[SPEC_MAX_HEADS];       /* bf16  [N_l, d_inner]: post-GELU state of level l */
+    uint64_t proj;                        /* fp32  [max rows, d_inner]: projected parent states */
+    uint64_t part_val, part_idx, part_ms; /* per-tile partial top-k lists and (max, sum-exp)  */
+    uint64_t logits;                      /* fp32 [max N_l, V]; only with SPEC_OPT_GEMM_IMPL=1 */
+    int32_t block_n[SPEC_MAX_HEADS];      /* vocabulary columns per head-GEMM tile            */
+    int32_t n_tiles[SPEC_MAX_HEADS];      /* vocabulary tiles per row of the head GEMM        */
+} spec_draft_layout_t;
+
+int spec_version(void);
+const char *spec_status_str(int status);
+/* cudaError_t / CUresult of the last failing CUDA call made by this library on this thread. */
+int spec_last_cuda_error(void);
+
+/* Host-only: validates and copies `w` (host), prepares host-side launch state.  The
+ * current CUDA device must be the one that owns the weight pointers. */
+int spec_create(spec_handle_t *out, const spec_weights_t *w);
+int spec_destroy(spec_handle_t h);
+int spec_set_option(spec_handle_t h, int option, int value);
+
+/* ---- draft (Sec. 3.1: multi-stage MLP emitting a tree of candidates; Sec. 4.1: branch
+ * topk[l] ways at head l, then prune the product tree to the K most confident) ----------
+ * For each sequence b: level 0 is (ctx_state[b], last_tok[b]); head l maps every node
+ * (parent state s, token t) to  s' = GELU(LayerNorm(a * Wp_l s + b * E_l[t])) rounded to
+ * bf16, logits = Wout_l s', and branches to the topk[l] largest logits (equal values:
+ * lower token id first) with score += logit - logsumexp(logits).  The K leaves with the
+ * best scores (equal scores: lower leaf index first) are returned in that order.
+ *   ctx_state  dev bf16 [B, d_base]   latest base-model state vector of each sequence
+ *   last_tok   dev int32 [B]          token just sampled from it
+ *   topk       host int32 [n_heads], 1 <= topk[l] <= SPEC_MAX_TOPK, prod <= SPEC_MAX_LEAVES
+ *   K          1 <= K <= prod topk
+ *   cand_tok   dev int32 [B, K, n_heads] (out), cand_logp dev fp32 [B, K] (out)
+ *   workspace  dev, 256-byte aligned, >= spec_draft_workspace_bytes(...)
+ */
+size_t spec_draft_workspace_bytes(spec_handle_t h, int B, const int32_t *topk, int K);
+int spec_draft_layout(spec_handle_t h, int B, const int32_t *topk, int K, spec_draft_layout_t *out /*host*/);
+int spec_draft(spec_handle_t h, const void *ctx_state, const int32_t *last_tok, int B, const int32_t *topk, int K,
+               int32_t *cand_tok, float *cand_logp, void *workspace, size_t workspace_bytes, void *cuda_stream);
+
+/* ---- verify (Sec. 1: accept the speculated tokens that match the base model's outputs;
+ * Sec. 3.1: score all candidates, keep the best; Sec. 5: at most n + 1 tokens per step) --
+ *   g[b,k,j]      = first index of the maximum of base_logits[b,k,j,:] (NaN never wins)
+ *   m[b,k]        = number of leading j < n with cand_tok[b,k,j] == g[b,k,j]
+ *   best_cand[b]  = lowest k attaining max_k m[b,k];  accept_len[b] = m[b,best];
+ *   next_tok[b]   = g[b,best,accept_len[b]]
+ *   cand_tok      dev int32 [B, K, n];  base_logits dev [B, K, n+1, V] of logits_dtype
+ *   accept_len, best_cand, next_tok  dev int32 [B] (out)
+ *   workspace     dev, 256-byte aligned, >= spec_verify_workspace_bytes(...); on return it
+ *                 holds the error word (offset 0) and g as int32 [B,K,n+1] at offset 256.
+ * Limits: K <= 65535, K * (n + 1) <= 12288.
+ */
+size_t spec_verify_workspace_bytes(int B, int K, int n, int V, int logits_dtype);
+int spec_verify(const int32_t *cand_tok, const void *base_logits, int logits_dtype, int B, int K, int n, int V,
+                int32_t *accept_len, int32_t *best_cand, int32_t *next_tok, void *workspace,
+                size_t workspace_bytes, void *cuda_stream);
+
+/* Per-kernel device times of the last spec_draft issued with SPEC_OPT_PROFILE = 1, in launch
+ * order: for every head (projection GEMM, mix/LayerNorm/GELU, head GEMM, merge/expand), then
+ * the prune kernel: 4 * n_heads + 1 values.  Blocks until that draft has finished.
+ *   ms_out host fp32 [max_count]; *count_out receives the number of values written. */
+int spec_profile_read(spec_handle_t h, float *ms_out, int max_count, int *count_out);
+
+/* Synchronises the stream, reads and clears the error word at the start of `workspace`
+ * (a draft or verify workspace) and returns it as a SPEC_* status. */
+int spec_poll_error(void *workspace, void *cuda_stream);
+
+/* ---- single steps, exported for parity tests and kernel benchmarks ---------------------
+ * spec_head_logits: logits[r, v] = sum_c head_l[v, c] * states[r, c] written in full
+ *   (fp32 [rows, V], dev) through the same tensor-core main loop as spec_draft.
+ * spec_head_topk: the fused form used inside spec_draft: per row the topk largest logits
+ *   (tok, dev int32 [rows, topk]) and their log-probabilities (logp, dev fp32 [rows, topk]);
+ *   full logits are never written.  workspace >= spec_head_workspace_bytes(...).
+ */
+size_t spec_head_workspace_bytes(spec_handle_t h, int rows, int topk);
+int spec_head_logits(spec_handle_t h, int level, const void *states /*dev bf16 [rows, d_inner]*/, int rows,
+                     float *logits, void *cuda_stream);
+int spec_head_topk(spec_handle_t h, int level, const void *states, int rows, int topk, int32_t *tok, float *logp,
+                   void *workspace, size_t workspace_bytes, void *cuda_stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SPEC_B200_H_ */

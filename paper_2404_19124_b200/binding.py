@@ -1,0 +1,294 @@
+"""Thin ctypes binding of libspec_b200.so (the C ABI declared in include/spec_b200.h).
+
+Argument marshalling only: every step of the draft / verify path runs inside the CUDA
+library.  PyTorch supplies device memory and streams.  There is no fallback: if the
+compiled library is missing, importing this module raises.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import List, Optional, Sequence
+
+import torch
+
+_PKG = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_PKG, "libspec_b200.so")
+
+MAX_HEADS, MAX_TOPK, MAX_LEAVES = 8, 8, 4096
+(SPEC_OK, SPEC_ERR_INVALID_ARG, SPEC_ERR_SHAPE, SPEC_ERR_WORKSPACE, SPEC_ERR_CUDA, SPEC_ERR_TOKEN_RANGE,
+ SPEC_ERR_TIMEOUT, SPEC_ERR_NO_DEVICE) = range(8)
+SPEC_BF16, SPEC_F32 = 0, 1
+SPEC_OPT_GEMM_IMPL, SPEC_OPT_HEAD_BLOCK_N, SPEC_OPT_PROJ_BLOCK_N, SPEC_OPT_PROFILE = 0, 1, 2, 3
+
+EXPORTS = [
+    "spec_version", "spec_status_str", "spec_last_cuda_error", "spec_create", "spec_destroy", "spec_set_option",
+    "spec_draft_workspace_bytes", "spec_draft_layout", "spec_draft", "spec_verify_workspace_bytes", "spec_verify",
+    "spec_profile_read", "spec_poll_error", "spec_head_workspace_bytes", "spec_head_logits", "spec_head_topk",
+]
+
+if not os.path.exists(LIB_PATH):
+    raise ImportError(
+        f"{LIB_PATH} is missing: build it with `python -m paper_2404_19124_b200.build` "
+        "(nvcc, sm_100a). There is no CPU or PyTorch fallback for the draft / verify path.")
+
+_lib = C.CDLL(LIB_PATH)
+
+
+class SpecWeightsC(C.Structure):
+    _fields_ = [
+        ("n_heads", C.c_int32), ("V", C.c_int32), ("d_base", C.c_int32), ("d_inner", C.c_int32),
+        ("emb", C.c_void_p * MAX_HEADS), ("proj", C.c_void_p * MAX_HEADS),
+        ("ln_gamma", C.c_void_p * MAX_HEADS), ("ln_beta", C.c_void_p * MAX_HEADS),
+        ("head", C.c_void_p * MAX_HEADS),
+        ("state_weight", C.c_float), ("emb_weight", C.c_float), ("ln_eps", C.c_float),
+    ]
+
+
+class SpecDraftLayoutC(C.Structure):
+    _fields_ = [
+        ("total_bytes", C.c_uint64), ("error_word", C.c_uint64),
+        ("tok", C.c_uint64 * (MAX_HEADS + 1)), ("score", C.c_uint64 * (MAX_HEADS + 1)),
+        ("state", C.c_uint64 * MAX_HEADS), ("proj", C.c_uint64),
+        ("part_val", C.c_uint64), ("part_idx", C.c_uint64), ("part_ms", C.c_uint64), ("logits", C.c_uint64),
+        ("block_n", C.c_int32 * MAX_HEADS), ("n_tiles", C.c_int32 * MAX_HEADS),
+    ]
+
+
+_lib.spec_version.restype = C.c_int
+_lib.spec_status_str.restype = C.c_char_p
+_lib.spec_status_str.argtypes = [C.c_int]
+_lib.spec_last_cuda_error.restype = C.c_int
+_lib.spec_create.argtypes = [C.POINTER(C.c_void_p), C.POINTER(SpecWeightsC)]
+_lib.spec_destroy.argtypes = [C.c_void_p]
+_lib.spec_set_option.argtypes = [C.c_void_p, C.c_int, C.c_int]
+_lib.spec_draft_workspace_bytes.restype = C.c_size_t
+_lib.spec_draft_workspace_bytes.argtypes = [C.c_void_p, C.c_int, C.POINTER(C.c_int32), C.c_int]
+_lib.spec_draft_layout.argtypes = [C.c_void_p, C.c_int, C.POINTER(C.c_int32), C.c_int, C.POINTER(SpecDraftLayoutC)]
+_lib.spec_draft.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int, C.POINTER(C.c_int32), C.c_int,
+                            C.c_void_p, C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]
+_lib.spec_verify_workspace_bytes.restype = C.c_size_t
+_lib.spec_verify_workspace_bytes.argtypes = [C.c_int] * 5
+_lib.spec_verify.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_int, C.c_int, C.c_int,
+                             C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]
+_lib.spec_poll_error.argtypes = [C.c_void_p, C.c_void_p]
+_lib.spec_profile_read.argtypes = [C.c_void_p, C.POINTER(C.c_float), C.c_int, C.POINTER(C.c_int)]
+_lib.spec_head_workspace_bytes.restype = C.c_size_t
+_lib.spec_head_workspace_bytes.argtypes = [C.c_void_p, C.c_int, C.c_int]
+_lib.spec_head_logits.argtypes = [C.c_void_p, C.c_int, C.c_void_p, C.c_int, C.c_void_p, C.c_void_p]
+_lib.spec_head_topk.argtypes = [C.c_void_p, C.c_int, C.c_void_p, C.c_int, C.c_int, C.c_void_p, C.c_void_p,
+                                C.c_void_p, C.c_size_t, C.c_void_p]
+
+
+class SpecError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        msg = _lib.spec_status_str(status).decode()
+        extra = f" (cuda error {_lib.spec_last_cuda_error()})" if status == SPEC_ERR_CUDA else ""
+        super().__init__(f"{where}: {msg}{extra}")
+        self.status = status
+
+
+def _check(status: int, where: str) -> None:
+    if status != SPEC_OK:
+        raise SpecError(status, where)
+
+
+def _ptr(t: Optional[torch.Tensor]):
+    return None if t is None else C.c_void_p(t.data_ptr())
+
+
+def _stream_ptr(stream: Optional[torch.cuda.Stream]):
+    s = torch.cuda.current_stream() if stream is None else stream
+    return C.c_void_p(s.cuda_stream)
+
+
+def _dev(t: torch.Tensor, dtype: torch.dtype, shape=None, name: str = "tensor") -> torch.Tensor:
+    if not t.is_cuda or t.dtype != dtype or not t.is_contiguous():
+        raise ValueError(f"{name} must be a contiguous CUDA tensor of {dtype}")
+    if shape is not None and tuple(t.shape) != tuple(shape):
+        raise ValueError(f"{name} must have shape {tuple(shape)}, got {tuple(t.shape)}")
+    return t
+
+
+def _topk_arr(topk: Sequence[int]):
+    return (C.c_int32 * len(topk))(*[int(x) for x in topk])
+
+
+def spec_version() -> int:
+    return int(_lib.spec_version())
+
+
+def spec_status_str(status: int) -> str:
+    return _lib.spec_status_str(int(status)).decode()
+
+
+class SpecHandle:
+    """Owns a spec_handle_t and keeps the weight tensors alive."""
+
+    def __init__(self, emb: List[torch.Tensor], proj: List[torch.Tensor], ln_gamma: List[torch.Tensor],
+                 ln_beta: List[torch.Tensor], head: List[torch.Tensor], state_weight: float, emb_weight: float,
+                 ln_eps: float = 1e-5):
+        n = len(head)
+        if not (1 <= n <= MAX_HEADS) or not all(len(x) == n for x in (emb, proj, ln_gamma, ln_beta)):
+            raise ValueError("need the same number (1..8) of emb / proj / ln_gamma / ln_beta / head tensors")
+        V, d_inner = head[0].shape
+        d_base = proj[0].shape[1]
+        w = SpecWeightsC()
+        w.n_heads, w.V, w.d_base, w.d_inner = n, V, d_base, d_inner
+        for l in range(n):
+            d_in = d_base if l == 0 else d_inner
+            w.emb[l] = _dev(emb[l], torch.bfloat16, (V, d_inner), f"emb[{l}]").data_ptr()
+            w.proj[l] = _dev(proj[l], torch.bfloat16, (d_inner, d_in), f"proj[{l}]").data_ptr()
+            w.ln_gamma[l] = _dev(ln_gamma[l], torch.float32, (d_inner,), f"ln_gamma[{l}]").data_ptr()
+            w.ln_beta[l] = _dev(ln_beta[l], torch.float32, (d_inner,), f"ln_beta[{l}]").data_ptr()
+            w.head[l] = _dev(head[l], torch.bfloat16, (V, d_inner), f"head[{l}]").data_ptr()
+        w.state_weight, w.emb_weight, w.ln_eps = state_weight, emb_weight, ln_eps
+        self._keep = (emb, proj, ln_gamma, ln_beta, head)
+        self.n_heads, self.V, self.d_base, self.d_inner = n, V, d_base, d_inner
+        self.device = head[0].device
+        self._h = C.c_void_p()
+        with torch.cuda.device(self.device):
+            _check(_lib.spec_create(C.byref(self._h), C.byref(w)), "spec_create")
+
+    def close(self) -> None:
+        if getattr(self, "_h", None) and self._h.value:
+            _lib.spec_destroy(self._h)
+            self._h = C.c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    @property
+    def ptr(self):
+        return self._h
+
+
+def spec_create(weights) -> SpecHandle:
+    """`weights`: an object with emb / proj / ln_gamma / ln_beta / head tensor lists (CUDA) and the scalars
+    state_weight, emb_weight, ln_eps (e.g. synth.SpecWeights moved to the GPU)."""
+    return SpecHandle(weights.emb, weights.proj, weights.ln_gamma, weights.ln_beta, weights.head,
+                      weights.state_weight, weights.emb_weight, weights.ln_eps)
+
+
+def spec_destroy(h: SpecHandle) -> None:
+    h.close()
+
+
+def spec_set_option(h: SpecHandle, option: int, value: int) -> None:
+    _check(_lib.spec_set_option(h.ptr, int(option), int(value)), "spec_set_option")
+
+
+def spec_draft_workspace_bytes(h: SpecHandle, B: int, topk: Sequence[int], K: int) -> int:
+    return int(_lib.spec_draft_workspace_bytes(h.ptr, int(B), _topk_arr(topk), int(K)))
+
+
+def spec_draft_layout(h: SpecHandle, B: int, topk: Sequence[int], K: int) -> SpecDraftLayoutC:
+    lay = SpecDraftLayoutC()
+    _check(_lib.spec_draft_layout(h.ptr, int(B), _topk_arr(topk), int(K), C.byref(lay)), "spec_draft_layout")
+    return lay
+
+
+def spec_draft(h: SpecHandle, ctx_state: torch.Tensor, last_tok: torch.Tensor, topk: Sequence[int], K: int,
+               cand_tok: Optional[torch.Tensor] = None, cand_logp: Optional[torch.Tensor] = None,
+               workspace: Optional[torch.Tensor] = None, stream: Optional[torch.cuda.Stream] = None):
+    """Enqueues one draft; returns (cand_tok [B,K,n] int32, cand_logp [B,K] fp32, workspace)."""
+    B = ctx_state.shape[0]
+    _dev(ctx_state, torch.bfloat16, (B, h.d_base), "ctx_state")
+    _dev(last_tok, torch.int32, (B,), "last_tok")
+    if len(topk) != h.n_heads:
+        raise SpecError(SPEC_ERR_SHAPE, "spec_draft: len(topk) != n_heads")
+    if cand_tok is None:
+        cand_tok = torch.empty((B, K, h.n_heads), dtype=torch.int32, device=h.device)
+    if cand_logp is None:
+        cand_logp = torch.empty((B, K), dtype=torch.float32, device=h.device)
+    _dev(cand_tok, torch.int32, (B, K, h.n_heads), "cand_tok")
+    _dev(cand_logp, torch.float32, (B, K), "cand_logp")
+    if workspace is None:
+        need = spec_draft_workspace_bytes(h, B, topk, K)
+        if need == 0:
+            raise SpecError(SPEC_ERR_SHAPE, "spec_draft_workspace_bytes")
+        workspace = torch.empty(need, dtype=torch.uint8, device=h.device)
+    _check(_lib.spec_draft(h.ptr, _ptr(ctx_state), _ptr(last_tok), B, _topk_arr(topk), int(K), _ptr(cand_tok),
+                           _ptr(cand_logp), _ptr(workspace), workspace.numel(), _stream_ptr(stream)), "spec_draft")
+    return cand_tok, cand_logp, workspace
+
+
+def spec_verify_workspace_bytes(B: int, K: int, n: int, V: int, logits_dtype: int) -> int:
+    return int(_lib.spec_verify_workspace_bytes(B, K, n, V, logits_dtype))
+
+
+def spec_verify(cand_tok: torch.Tensor, base_logits: torch.Tensor, accept_len: Optional[torch.Tensor] = None,
+                best_cand: Optional[torch.Tensor] = None, next_tok: Optional[torch.Tensor] = None,
+                workspace: Optional[torch.Tensor] = None, stream: Optional[torch.cuda.Stream] = None):
+    """Enqueues one verification; returns (accept_len, best_cand, next_tok, workspace), int32 [B] each."""
+    B, K, n = cand_tok.shape
+    _dev(cand_tok, torch.int32, name="cand_tok")
+    if base_logits.dtype == torch.bfloat16:
+        dt = SPEC_BF16
+    elif base_logits.dtype == torch.float32:
+        dt = SPEC_F32
+    else:
+        raise ValueError("base_logits must be bf16 or fp32")
+    V = base_logits.shape[-1]
+    _dev(base_logits, base_logits.dtype, (B, K, n + 1, V), "base_logits")
+    dev = cand_tok.device
+    outs = []
+    for t, name in ((accept_len, "accept_len"), (best_cand, "best_cand"), (next_tok, "next_tok")):
+        if t is None:
+            t = torch.empty(B, dtype=torch.int32, device=dev)
+        outs.append(_dev(t, torch.int32, (B,), name))
+    if workspace is None:
+        need = spec_verify_workspace_bytes(B, K, n, V, dt)
+        if need == 0:
+            raise SpecError(SPEC_ERR_SHAPE, "spec_verify_workspace_bytes")
+        workspace = torch.empty(need, dtype=torch.uint8, device=dev)
+    _check(_lib.spec_verify(_ptr(cand_tok), _ptr(base_logits), dt, B, K, n, V, _ptr(outs[0]), _ptr(outs[1]),
+                            _ptr(outs[2]), _ptr(workspace), workspace.numel(), _stream_ptr(stream)), "spec_verify")
+    return outs[0], outs[1], outs[2], workspace
+
+
+def spec_profile_read(h: SpecHandle) -> List[float]:
+    """Per-kernel milliseconds of the last profiled spec_draft (see SPEC_OPT_PROFILE)."""
+    buf = (C.c_float * 64)()
+    cnt = C.c_int(0)
+    _check(_lib.spec_profile_read(h.ptr, buf, 64, C.byref(cnt)), "spec_profile_read")
+    return [float(buf[i]) for i in range(cnt.value)]
+
+
+def spec_poll_error(workspace: torch.Tensor, stream: Optional[torch.cuda.Stream] = None) -> int:
+    return int(_lib.spec_poll_error(_ptr(workspace), _stream_ptr(stream)))
+
+
+def spec_head_workspace_bytes(h: SpecHandle, rows: int, topk: int) -> int:
+    return int(_lib.spec_head_workspace_bytes(h.ptr, int(rows), int(topk)))
+
+
+def spec_head_logits(h: SpecHandle, level: int, states: torch.Tensor, logits: Optional[torch.Tensor] = None,
+                     stream: Optional[torch.cuda.Stream] = None) -> torch.Tensor:
+    rows = states.shape[0]
+    _dev(states, torch.bfloat16, (rows, h.d_inner), "states")
+    if logits is None:
+        logits = torch.empty((rows, h.V), dtype=torch.float32, device=h.device)
+    _dev(logits, torch.float32, (rows, h.V), "logits")
+    _check(_lib.spec_head_logits(h.ptr, int(level), _ptr(states), rows, _ptr(logits), _stream_ptr(stream)),
+           "spec_head_logits")
+    return logits
+
+
+def spec_head_topk(h: SpecHandle, level: int, states: torch.Tensor, topk: int, tok: Optional[torch.Tensor] = None,
+                   logp: Optional[torch.Tensor] = None, workspace: Optional[torch.Tensor] = None,
+                   stream: Optional[torch.cuda.Stream] = None):
+    rows = states.shape[0]
+    _dev(states, torch.bfloat16, (rows, h.d_inner), "states")
+    if tok is None:
+        tok = torch.empty((rows, topk), dtype=torch.int32, device=h.device)
+    if logp is None:
+        logp = torch.empty((rows, topk), dtype=torch.float32, device=h.device)
+    if workspace is None:
+        workspace = torch.empty(spec_head_workspace_bytes(h, rows, topk), dtype=torch.uint8, device=h.device)
+    _check(_lib.spec_head_topk(h.ptr, int(level), _ptr(states), rows, int(topk), _ptr(tok), _ptr(logp),
+                               _ptr(workspace), workspace.numel(), _stream_ptr(stream)), "spec_head_topk")
+    return tok, logp, workspace

@@ -1,0 +1,425 @@
+// C ABI of libspec_b200: host-side validation, workspace layout and the launch sequences of
+// spec_draft / spec_verify (declared and documented in include/spec_b200.h).
+#include <new>
+#include <string.h>
+
+#include "spec_common.cuh"
+
+namespace spec {
+
+static thread_local int g_last_cuda_error = 0;
+void set_last_cuda_error(int e) { g_last_cuda_error = e; }
+
+int num_sms() {
+    static int cached[64] = {};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return kNumSMsFallback;
+    if (cached[dev] == 0) {
+        int n = 0;
+        if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0)
+            n = kNumSMsFallback;
+        cached[dev] = n;
+    }
+    return cached[dev];
+}
+
+}  // namespace spec
+
+using namespace spec;
+
+constexpr int kMaxProfEvents = 4 * SPEC_MAX_HEADS + 2;
+
+struct spec_handle_s {
+    spec_weights_t w;
+    int gemm_impl;
+    int head_block_n;
+    int proj_block_n;
+    int profile;
+    int prof_count;                        // events recorded by the last profiled draft
+    cudaEvent_t prof_ev[kMaxProfEvents];   // created when profiling is switched on
+};
+
+namespace {
+
+size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+int d_in_of(const spec_weights_t &w, int l) { return l == 0 ? w.d_base : w.d_inner; }
+
+// Shapes of one draft call and where everything lives in the workspace.
+struct DraftPlan {
+    int n;
+    int N[SPEC_MAX_HEADS + 1];   // nodes per level
+    int L;
+    spec_draft_layout_t lay;
+    int proj_block_n[SPEC_MAX_HEADS];
+};
+
+int head_block_n_for(const spec_handle_s *h, int rows) {
+    if (h->head_block_n > 0) return h->head_block_n;
+    return choose_block_n(rows, h->w.V, num_sms(), rows > 128);
+}
+
+int proj_block_n_for(const spec_handle_s *h, int rows) {
+    if (h->proj_block_n > 0) return h->proj_block_n;
+    return choose_block_n(rows, h->w.d_inner, num_sms(), rows > 128);
+}
+
+int make_draft_plan(const spec_handle_s *h, int B, const int32_t *topk, int K, DraftPlan *p) {
+    if (!h || !topk || !p) return SPEC_ERR_INVALID_ARG;
+    if (B <= 0 || K <= 0) return SPEC_ERR_INVALID_ARG;
+    const spec_weights_t &w = h->w;
+    memset(p, 0, sizeof(*p));
+    p->n = w.n_heads;
+    long long nodes = B, leaves = 1;
+    p->N[0] = B;
+    for (int l = 0; l < p->n; ++l) {
+        if (topk[l] < 1 || topk[l] > SPEC_MAX_TOPK || topk[l] > w.V) return SPEC_ERR_SHAPE;
+        leaves *= topk[l];
+        nodes *= topk[l];
+        if (leaves > SPEC_MAX_LEAVES || nodes > (1ll << 24)) return SPEC_ERR_SHAPE;
+        p->N[l + 1] = (int)nodes;
+    }
+    if (K > leaves) return SPEC_ERR_SHAPE;
+    p->L = (int)leaves;
+
+    spec_draft_layout_t &y = p->lay;
+    size_t off = kWsAlign;   // error word lives at offset 0
+    y.error_word = 0;
+    for (int l = 1; l <= p->n; ++l) {
+        y.tok[l] = off;
+        off = align_up(off + sizeof(int32_t) * (size_t)p->N[l], kWsAlign);
+        y.score[l] = off;
+        off = align_up(off + sizeof(float) * (size_t)p->N[l], kWsAlign);
+    }
+    int max_parent_rows = B;
+    size_t max_part_units = 0;
+    int max_rows = 0;
+    for (int l = 0; l < p->n; ++l) {
+        y.state[l] = off;
+        off = align_up(off + 2 * (size_t)p->N[l] * w.d_inner, kWsAlign);
+        if (l > 0 && p->N[l - 1] > max_parent_rows) max_parent_rows = p->N[l - 1];
+        const int bn = head_block_n_for(h, p->N[l]);
+        y.block_n[l] = bn;
+        y.n_tiles[l] = (w.V + bn - 1) / bn;
+        const size_t units = (size_t)p->N[l] * y.n_tiles[l];
+        if (units > max_part_units) max_part_units = units;
+        if (p->N[l] > max_rows) max_rows = p->N[l];
+        p->proj_block_n[l] = proj_block_n_for(h, l == 0 ? B : p->N[l - 1]);
+    }
+    y.proj = off;
+    off = align_up(off + sizeof(float) * (size_t)max_parent_rows * w.d_inner, kWsAlign);
+    y.part_val = off;
+    off = align_up(off + sizeof(float) * max_part_units * SPEC_MAX_TOPK, kWsAlign);
+    y.part_idx = off;
+    off = align_up(off + sizeof(int32_t) * max_part_units * SPEC_MAX_TOPK, kWsAlign);
+    y.part_ms = off;
+    off = align_up(off + sizeof(float) * max_part_units * 2, kWsAlign);
+    y.logits = off;
+    if (h->gemm_impl == 1) off = align_up(off + sizeof(float) * (size_t)max_rows * w.V, kWsAlign);
+    y.total_bytes = off;
+    return SPEC_OK;
+}
+
+// One contraction through whichever implementation the handle selects.
+int run_gemm_store(const spec_handle_s *h, const void *A, const void *Bm, int M, int N, int Kd, int block_n,
+                   float *out, int32_t *err, cudaStream_t st) {
+    if (h->gemm_impl == 1) return launch_gemm_simt(A, Bm, M, N, Kd, out, N, st);
+    GemmEpilogue e{};
+    e.mode = 0;
+    e.out = out;
+    e.ldc = N;
+    return launch_gemm_tc(A, Bm, M, N, Kd, block_n, e, err, st);
+}
+
+int run_head_partials(const spec_handle_s *h, const void *states, const void *Wout, int rows, int block_n, int topk,
+                      float *part_val, int32_t *part_idx, float *part_ms, float *logits_scratch, int32_t *err,
+                      cudaStream_t st) {
+    const spec_weights_t &w = h->w;
+    if (h->gemm_impl == 1) {
+        int rc = launch_gemm_simt(states, Wout, rows, w.V, w.d_inner, logits_scratch, w.V, st);
+        if (rc != SPEC_OK) return rc;
+        return launch_partials_from_logits(logits_scratch, rows, w.V, block_n, topk, part_val, part_idx, part_ms, st);
+    }
+    GemmEpilogue e{};
+    e.mode = 1;
+    e.part_val = part_val;
+    e.part_idx = part_idx;
+    e.part_ms = part_ms;
+    e.topk = topk;
+    return launch_gemm_tc(states, Wout, rows, w.V, w.d_inner, block_n, e, err, st);
+}
+
+}  // namespace
+
+extern "C" {
+
+int spec_version(void) { return 1; }
+
+const char *spec_status_str(int s) {
+    switch (s) {
+        case SPEC_OK: return "ok";
+        case SPEC_ERR_INVALID_ARG: return "invalid argument";
+        case SPEC_ERR_SHAPE: return "unsupported shape";
+        case SPEC_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
+        case SPEC_ERR_CUDA: return "CUDA call failed";
+        case SPEC_ERR_TOKEN_RANGE: return "token id outside the vocabulary";
+        case SPEC_ERR_TIMEOUT: return "bounded wait inside a kernel ran out";
+        case SPEC_ERR_NO_DEVICE: return "no usable CUDA device";
+        default: return "unknown status";
+    }
+}
+
+int spec_last_cuda_error(void) { return g_last_cuda_error; }
+
+int spec_create(spec_handle_t *out, const spec_weights_t *w) {
+    if (!out || !w) return SPEC_ERR_INVALID_ARG;
+    *out = nullptr;
+    if (w->n_heads < 1 || w->n_heads > SPEC_MAX_HEADS || w->V < 1 || w->d_base < 8 || w->d_inner < 8)
+        return SPEC_ERR_SHAPE;
+    if (w->d_base % 8 != 0 || w->d_inner % 8 != 0) return SPEC_ERR_SHAPE;   // 16-byte rows for TMA and vector loads
+    for (int l = 0; l < w->n_heads; ++l) {
+        const void *ptrs[5] = {w->emb[l], w->proj[l], w->ln_gamma[l], w->ln_beta[l], w->head[l]};
+        for (const void *q : ptrs) {
+            if (!q) return SPEC_ERR_INVALID_ARG;
+            if ((uintptr_t)q & 15) return SPEC_ERR_INVALID_ARG;
+        }
+    }
+    if (!(w->ln_eps > 0.0f)) return SPEC_ERR_INVALID_ARG;
+    int count = 0;
+    if (cudaGetDeviceCount(&count) != cudaSuccess || count <= 0) {
+        (void)cudaGetLastError();
+        return SPEC_ERR_NO_DEVICE;
+    }
+    int dev = 0, major = 0;
+    SPEC_CUDA_TRY(cudaGetDevice(&dev));
+    SPEC_CUDA_TRY(cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev));
+    if (major != 10) return SPEC_ERR_NO_DEVICE;
+    spec_handle_s *h = new (std::nothrow) spec_handle_s();
+    if (!h) return SPEC_ERR_INVALID_ARG;
+    h->w = *w;
+    h->gemm_impl = 0;
+    h->head_block_n = 0;
+    h->proj_block_n = 0;
+    h->profile = 0;
+    h->prof_count = 0;
+    for (cudaEvent_t &e : h->prof_ev) e = nullptr;
+    *out = h;
+    return SPEC_OK;
+}
+
+int spec_destroy(spec_handle_t h) {
+    if (h)
+        for (cudaEvent_t e : h->prof_ev)
+            if (e) cudaEventDestroy(e);
+    delete h;
+    return SPEC_OK;
+}
+
+int spec_set_option(spec_handle_t h, int option, int value) {
+    if (!h) return SPEC_ERR_INVALID_ARG;
+    switch (option) {
+        case SPEC_OPT_GEMM_IMPL:
+            if (value != 0 && value != 1) return SPEC_ERR_INVALID_ARG;
+            h->gemm_impl = value;
+            return SPEC_OK;
+        case SPEC_OPT_HEAD_BLOCK_N:
+        case SPEC_OPT_PROJ_BLOCK_N:
+            if (value != 0 && (value < 32 || value > 256 || value % 32 != 0)) return SPEC_ERR_INVALID_ARG;
+            (option == SPEC_OPT_HEAD_BLOCK_N ? h->head_block_n : h->proj_block_n) = value;
+            return SPEC_OK;
+        case SPEC_OPT_PROFILE:
+            if (value != 0 && value != 1) return SPEC_ERR_INVALID_ARG;
+            if (value == 1)
+                for (cudaEvent_t &e : h->prof_ev)
+                    if (!e) SPEC_CUDA_TRY(cudaEventCreate(&e));
+            h->profile = value;
+            h->prof_count = 0;
+            return SPEC_OK;
+        default:
+            return SPEC_ERR_INVALID_ARG;
+    }
+}
+
+int spec_profile_read(spec_handle_t h, float *ms_out, int max_count, int *count_out) {
+    if (!h || !ms_out || !count_out || max_count < 0) return SPEC_ERR_INVALID_ARG;
+    *count_out = 0;
+    if (h->prof_count < 2) return SPEC_OK;
+    SPEC_CUDA_TRY(cudaEventSynchronize(h->prof_ev[h->prof_count - 1]));
+    for (int i = 0; i + 1 < h->prof_count && i < max_count; ++i) {
+        SPEC_CUDA_TRY(cudaEventElapsedTime(&ms_out[i], h->prof_ev[i], h->prof_ev[i + 1]));
+        *count_out = i + 1;
+    }
+    return SPEC_OK;
+}
+
+size_t spec_draft_workspace_bytes(spec_handle_t h, int B, const int32_t *topk, int K) {
+    DraftPlan p;
+    if (make_draft_plan(h, B, topk, K, &p) != SPEC_OK) return 0;
+    return (size_t)p.lay.total_bytes;
+}
+
+int spec_draft_layout(spec_handle_t h, int B, const int32_t *topk, int K, spec_draft_layout_t *out) {
+    if (!out) return SPEC_ERR_INVALID_ARG;
+    DraftPlan p;
+    int rc = make_draft_plan(h, B, topk, K, &p);
+    if (rc != SPEC_OK) return rc;
+    *out = p.lay;
+    return SPEC_OK;
+}
+
+int spec_draft(spec_handle_t h, const void *ctx_state, const int32_t *last_tok, int B, const int32_t *topk, int K,
+               int32_t *cand_tok, float *cand_logp, void *workspace, size_t workspace_bytes, void *cuda_stream) {
+    if (!h || !ctx_state || !last_tok || !topk || !cand_tok || !cand_logp) return SPEC_ERR_INVALID_ARG;
+    if ((uintptr_t)ctx_state & 15) return SPEC_ERR_INVALID_ARG;
+    DraftPlan p;
+    int rc = make_draft_plan(h, B, topk, K, &p);
+    if (rc != SPEC_OK) return rc;
+    if (!workspace || ((uintptr_t)workspace % kWsAlign) != 0 || workspace_bytes < p.lay.total_bytes)
+        return SPEC_ERR_WORKSPACE;
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    const spec_weights_t &w = h->w;
+    char *ws = (char *)workspace;
+    int32_t *err = (int32_t *)(ws + p.lay.error_word);
+    SPEC_CUDA_TRY(cudaMemsetAsync(err, 0, sizeof(int32_t), st));
+
+    int nev = 0;
+    h->prof_count = 0;
+#define SPEC_PROF_MARK()                                                     \
+    do {                                                                     \
+        if (h->profile) SPEC_CUDA_TRY(cudaEventRecord(h->prof_ev[nev++], st)); \
+    } while (0)
+    SPEC_PROF_MARK();
+
+    float *P = (float *)(ws + p.lay.proj);
+    float *part_val = (float *)(ws + p.lay.part_val);
+    int32_t *part_idx = (int32_t *)(ws + p.lay.part_idx);
+    float *part_ms = (float *)(ws + p.lay.part_ms);
+    float *logits_scratch = (float *)(ws + p.lay.logits);
+
+    for (int l = 0; l < p.n; ++l) {
+        const int rows = p.N[l];
+        const int parent_rows = l == 0 ? B : p.N[l - 1];
+        const void *parent_states = l == 0 ? ctx_state : (const void *)(ws + p.lay.state[l - 1]);
+        const int32_t *tok_l = l == 0 ? last_tok : (const int32_t *)(ws + p.lay.tok[l]);
+        const float *score_l = l == 0 ? nullptr : (const float *)(ws + p.lay.score[l]);
+        void *S = ws + p.lay.state[l];
+        // projection of every distinct parent state: P = S_parent * Wp^T
+        rc = run_gemm_store(h, parent_states, w.proj[l], parent_rows, w.d_inner, d_in_of(w, l), p.proj_block_n[l], P,
+                            err, st);
+        if (rc != SPEC_OK) return rc;
+        SPEC_PROF_MARK();
+        // gather + mix + LayerNorm + GELU -> bf16 state of every node of this level
+        rc = launch_mix_ln_gelu(P, w.emb[l], tok_l, w.ln_gamma[l], w.ln_beta[l], rows, w.d_inner, w.V,
+                                l == 0 ? 1 : topk[l - 1], w.state_weight, w.emb_weight, w.ln_eps, S, err, st);
+        if (rc != SPEC_OK) return rc;
+        SPEC_PROF_MARK();
+        // vocabulary head with the fused per-tile top-k / log-sum-exp epilogue
+        rc = run_head_partials(h, S, w.head[l], rows, p.lay.block_n[l], topk[l], part_val, part_idx, part_ms,
+                               logits_scratch, err, st);
+        if (rc != SPEC_OK) return rc;
+        SPEC_PROF_MARK();
+        // fold the partials, branch: children (token, cumulative score) of every node
+        rc = launch_merge_expand(part_val, part_idx, part_ms, rows, p.lay.n_tiles[l], topk[l], score_l,
+                                 (int32_t *)(ws + p.lay.tok[l + 1]), (float *)(ws + p.lay.score[l + 1]), 0, st);
+        if (rc != SPEC_OK) return rc;
+        SPEC_PROF_MARK();
+    }
+    PruneArgs pa{};
+    pa.n = p.n;
+    for (int l = 0; l < p.n; ++l) {
+        pa.tok[l] = (const int32_t *)(ws + p.lay.tok[l + 1]);
+        pa.topk[l] = topk[l];
+    }
+    rc = launch_prune((const float *)(ws + p.lay.score[p.n]), pa, B, p.L, K, cand_tok, cand_logp, st);
+    if (rc != SPEC_OK) return rc;
+    SPEC_PROF_MARK();
+#undef SPEC_PROF_MARK
+    h->prof_count = nev;
+    return SPEC_OK;
+}
+
+size_t spec_verify_workspace_bytes(int B, int K, int n, int V, int logits_dtype) {
+    if (B <= 0 || K <= 0 || n <= 0 || V <= 0) return 0;
+    if (logits_dtype != SPEC_BF16 && logits_dtype != SPEC_F32) return 0;
+    if ((long long)B * K * (n + 1) > (1ll << 30)) return 0;
+    return make_verify_plan(B, K, n, V, logits_dtype).total;
+}
+
+int spec_verify(const int32_t *cand_tok, const void *base_logits, int logits_dtype, int B, int K, int n, int V,
+                int32_t *accept_len, int32_t *best_cand, int32_t *next_tok, void *workspace, size_t workspace_bytes,
+                void *cuda_stream) {
+    if (!cand_tok || !base_logits || !accept_len || !best_cand || !next_tok) return SPEC_ERR_INVALID_ARG;
+    if (B <= 0 || K <= 0 || n <= 0 || V <= 0) return SPEC_ERR_INVALID_ARG;
+    if (logits_dtype != SPEC_BF16 && logits_dtype != SPEC_F32) return SPEC_ERR_INVALID_ARG;
+    if (K > 65535 || (long long)K * (n + 1) > 12288 || n > 32767) return SPEC_ERR_SHAPE;
+    if ((long long)B * K * (n + 1) > (1ll << 30)) return SPEC_ERR_SHAPE;
+    if (((uintptr_t)base_logits % (logits_dtype == SPEC_BF16 ? 2 : 4)) != 0) return SPEC_ERR_INVALID_ARG;
+    const VerifyPlan plan = make_verify_plan(B, K, n, V, logits_dtype);
+    if (!workspace || ((uintptr_t)workspace % kWsAlign) != 0 || workspace_bytes < plan.total)
+        return SPEC_ERR_WORKSPACE;
+    return launch_verify(cand_tok, base_logits, logits_dtype, B, K, n, V, accept_len, best_cand, next_tok, workspace,
+                         plan, (cudaStream_t)cuda_stream);
+}
+
+int spec_poll_error(void *workspace, void *cuda_stream) {
+    if (!workspace) return SPEC_ERR_INVALID_ARG;
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    int32_t word = 0;
+    SPEC_CUDA_TRY(cudaMemcpyAsync(&word, workspace, sizeof(word), cudaMemcpyDeviceToHost, st));
+    SPEC_CUDA_TRY(cudaStreamSynchronize(st));
+    if (word != 0) {
+        SPEC_CUDA_TRY(cudaMemsetAsync(workspace, 0, sizeof(word), st));
+        SPEC_CUDA_TRY(cudaStreamSynchronize(st));
+    }
+    return (int)word;
+}
+
+size_t spec_head_workspace_bytes(spec_handle_t h, int rows, int topk) {
+    if (!h || rows <= 0 || topk < 1 || topk > SPEC_MAX_TOPK) return 0;
+    const int bn = head_block_n_for(h, rows);
+    const size_t units = (size_t)rows * ((h->w.V + bn - 1) / bn);
+    size_t off = kWsAlign;
+    off = align_up(off + sizeof(float) * units * SPEC_MAX_TOPK, kWsAlign);
+    off = align_up(off + sizeof(int32_t) * units * SPEC_MAX_TOPK, kWsAlign);
+    off = align_up(off + sizeof(float) * units * 2, kWsAlign);
+    if (h->gemm_impl == 1) off = align_up(off + sizeof(float) * (size_t)rows * h->w.V, kWsAlign);
+    return off;
+}
+
+int spec_head_logits(spec_handle_t h, int level, const void *states, int rows, float *logits, void *cuda_stream) {
+    if (!h || !states || !logits || rows <= 0) return SPEC_ERR_INVALID_ARG;
+    if (level < 0 || level >= h->w.n_heads) return SPEC_ERR_SHAPE;
+    if ((uintptr_t)states & 15) return SPEC_ERR_INVALID_ARG;
+    return run_gemm_store(h, states, h->w.head[level], rows, h->w.V, h->w.d_inner, head_block_n_for(h, rows), logits,
+                          nullptr, (cudaStream_t)cuda_stream);
+}
+
+int spec_head_topk(spec_handle_t h, int level, const void *states, int rows, int topk, int32_t *tok, float *logp,
+                   void *workspace, size_t workspace_bytes, void *cuda_stream) {
+    if (!h || !states || !tok || !logp || rows <= 0) return SPEC_ERR_INVALID_ARG;
+    if (level < 0 || level >= h->w.n_heads || topk < 1 || topk > SPEC_MAX_TOPK || topk > h->w.V) return SPEC_ERR_SHAPE;
+    if ((uintptr_t)states & 15) return SPEC_ERR_INVALID_ARG;
+    const size_t need = spec_head_workspace_bytes(h, rows, topk);
+    if (!workspace || ((uintptr_t)workspace % kWsAlign) != 0 || workspace_bytes < need) return SPEC_ERR_WORKSPACE;
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    const int bn = head_block_n_for(h, rows);
+    const int n_tiles = (h->w.V + bn - 1) / bn;
+    const size_t units = (size_t)rows * n_tiles;
+    char *ws = (char *)workspace;
+    int32_t *err = (int32_t *)ws;
+    SPEC_CUDA_TRY(cudaMemsetAsync(err, 0, sizeof(int32_t), st));
+    size_t off = kWsAlign;
+    float *part_val = (float *)(ws + off);
+    off = align_up(off + sizeof(float) * units * SPEC_MAX_TOPK, kWsAlign);
+    int32_t *part_idx = (int32_t *)(ws + off);
+    off = align_up(off + sizeof(int32_t) * units * SPEC_MAX_TOPK, kWsAlign);
+    float *part_ms = (float *)(ws + off);
+    off = align_up(off + sizeof(float) * units * 2, kWsAlign);
+    float *logits_scratch = (float *)(ws + off);
+    int rc = run_head_partials(h, states, h->w.head[level], rows, bn, topk, part_val, part_idx, part_ms,
+                               logits_scratch, err, st);
+    if (rc != SPEC_OK) return rc;
+    return launch_merge_expand(part_val, part_idx, part_ms, rows, n_tiles, topk, nullptr, tok, logp, 0, st);
+}
+
+}  // extern "C"

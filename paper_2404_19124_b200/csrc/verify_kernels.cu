@@ -1,0 +1,223 @@
+// Greedy multi-candidate verification (Sec. 1, Sec. 3.1, Sec. 5 of arXiv 2404.19124):
+// a bandwidth-bound streaming arg-max over every row of the base model's logits followed by
+// the longest-matching-prefix / best-candidate reduction.
+//
+// Kernel 1 (verify_argmax_kernel): the B*K*(n+1) rows are cut into (row, chunk) work units,
+//   one warp per unit, 128-bit streaming loads with four loads in flight per lane.  For bf16
+//   the running maximum is taken on packed pairs (max.bf16x2), the element index is only
+//   resolved when a vector beats the lane's current best, so the common case costs about one
+//   ALU operation per element.  Each unit writes one (value, index) partial.
+// Kernel 2 (verify_accept_kernel): one CTA per sequence folds the partials of its K*(n+1)
+//   rows into g[b,k,j], counts the matching prefix of every candidate and picks the best one.
+#include <float.h>
+
+#include "spec_common.cuh"
+
+namespace spec {
+
+namespace {
+
+constexpr int kArgmaxThreads = 256;
+constexpr int kWarpsPerBlock = kArgmaxThreads / 32;
+constexpr int kIdxNone = 0x7fffffff;
+
+__device__ __forceinline__ uint32_t max_bf16x2(uint32_t a, uint32_t b) {
+    uint32_t d;
+    asm("max.bf16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));   // a NaN operand is dropped
+    return d;
+}
+
+__device__ __forceinline__ uint4 ld_stream(const uint4 *p) {
+    uint4 v;
+    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+                 : "l"(p));
+    return v;
+}
+
+// best/idx: the lane's running (maximum, first index).  `base` is the index of element 0 of v.
+__device__ __forceinline__ void consume_bf16(const uint4 &v, int base, float &best, int &idx) {
+    uint32_t m2 = max_bf16x2(max_bf16x2(v.x, v.y), max_bf16x2(v.z, v.w));
+    float mx = fmaxf(__uint_as_float(m2 << 16), __uint_as_float(m2 & 0xffff0000u));
+    if (mx > best) {   // rare after the first few vectors
+        best = mx;
+        const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+        int pos = 7;
+#pragma unroll
+        for (int i = 3; i >= 0; --i) {
+            if (__uint_as_float(w[i] & 0xffff0000u) == mx) pos = 2 * i + 1;
+            if (__uint_as_float(w[i] << 16) == mx) pos = 2 * i;
+        }
+        idx = base + pos;
+    }
+}
+
+__device__ __forceinline__ void consume_f32(const uint4 &v, int base, float &best, int &idx) {
+    const float f[4] = {__uint_as_float(v.x), __uint_as_float(v.y), __uint_as_float(v.z), __uint_as_float(v.w)};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        if (f[i] > best) {
+            best = f[i];
+            idx = base + i;
+        }
+    }
+}
+
+// (value desc, index asc) combine across the warp.
+__device__ __forceinline__ void warp_argmax(float &best, int &idx) {
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) {
+        float ob = __shfl_xor_sync(0xffffffffu, best, off);
+        int oi = __shfl_xor_sync(0xffffffffu, idx, off);
+        if (ob > best || (ob == best && oi < idx)) {
+            best = ob;
+            idx = oi;
+        }
+    }
+}
+
+template <bool kBf16, bool kVector>
+__global__ void __launch_bounds__(kArgmaxThreads)
+verify_argmax_kernel(const void *__restrict__ logits, int rows, int V, int chunk_elems, int chunks,
+                     float *__restrict__ pval, int32_t *__restrict__ pidx) {
+    const int lane = threadIdx.x & 31;
+    const long long unit = (long long)blockIdx.x * kWarpsPerBlock + (threadIdx.x >> 5);
+    if (unit >= (long long)rows * chunks) return;
+    const int row = (int)(unit / chunks), chunk = (int)(unit - (long long)row * chunks);
+    const int begin = chunk * chunk_elems;
+    const int count = min(chunk_elems, V - begin);
+    constexpr int kEsz = kBf16 ? 2 : 4;
+    const char *rp = (const char *)logits + ((size_t)row * V + begin) * kEsz;
+
+    float best = -INFINITY;
+    int idx = kIdxNone;
+    if (kVector) {
+        constexpr int kEpv = 16 / kEsz;
+        const uint4 *vp = (const uint4 *)rp;
+        const int nvec = count / kEpv;   // exact: V and chunk_elems are multiples of kEpv on this path
+        for (int v0 = lane; v0 < nvec; v0 += 128) {
+            uint4 q[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u)
+                if (v0 + 32 * u < nvec) q[u] = ld_stream(vp + v0 + 32 * u);
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                if (v0 + 32 * u < nvec) {
+                    const int base = begin + (v0 + 32 * u) * kEpv;
+                    if (kBf16) consume_bf16(q[u], base, best, idx);
+                    else consume_f32(q[u], base, best, idx);
+                }
+            }
+        }
+    } else {
+        for (int i = lane; i < count; i += 32) {
+            float x = kBf16 ? bf16_bits_to_float(((const uint16_t *)rp)[i]) : ((const float *)rp)[i];
+            if (x > best) {
+                best = x;
+                idx = begin + i;
+            }
+        }
+    }
+    warp_argmax(best, idx);
+    if (lane == 0) {
+        pval[unit] = best;
+        pidx[unit] = idx;
+    }
+}
+
+__global__ void __launch_bounds__(128)
+verify_accept_kernel(const int32_t *__restrict__ cand_tok, const float *__restrict__ pval,
+                     const int32_t *__restrict__ pidx, int K, int n, int chunks, int32_t *__restrict__ g_out,
+                     int32_t *__restrict__ accept_len, int32_t *__restrict__ best_cand,
+                     int32_t *__restrict__ next_tok, int32_t *err) {
+    extern __shared__ int32_t g_s[];   // [K * (n + 1)]
+    __shared__ unsigned int key_s;
+    const int b = blockIdx.x, rows_b = K * (n + 1);
+    if (threadIdx.x == 0) {
+        key_s = 0u;
+        if (b == 0 && err != nullptr) *err = 0;
+    }
+    for (int r = threadIdx.x; r < rows_b; r += blockDim.x) {
+        const size_t u0 = ((size_t)b * rows_b + r) * chunks;
+        float best = -INFINITY;
+        int arg = 0;   // a row without any value above -inf (all NaN) yields 0
+        for (int c = 0; c < chunks; ++c) {
+            const float v = pval[u0 + c];
+            if (v > best) {   // chunks ascend, so the first maximum wins
+                best = v;
+                arg = pidx[u0 + c];
+            }
+        }
+        g_s[r] = arg;
+        g_out[(size_t)b * rows_b + r] = arg;
+    }
+    __syncthreads();
+    for (int k = threadIdx.x; k < K; k += blockDim.x) {
+        const int32_t *c = cand_tok + ((size_t)b * K + k) * n;
+        const int32_t *gk = g_s + k * (n + 1);
+        int m = 0;
+        while (m < n && c[m] == gk[m]) ++m;
+        // longest prefix first, then the lowest candidate index
+        atomicMax(&key_s, ((unsigned)m << 16) | (unsigned)(0xffff - k));
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        const int m = (int)(key_s >> 16), k = 0xffff - (int)(key_s & 0xffffu);
+        accept_len[b] = m;
+        best_cand[b] = k;
+        next_tok[b] = g_s[k * (n + 1) + m];
+    }
+}
+
+size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+}  // namespace
+
+VerifyPlan make_verify_plan(int B, int K, int n, int V, int dtype) {
+    VerifyPlan p{};
+    p.rows = B * K * (n + 1);
+    const int esz = dtype == SPEC_BF16 ? 2 : 4;
+    const int gran = 32 * 4 * (16 / esz);   // elements one warp covers per loop trip
+    const long long target_units = (long long)num_sms() * 64 * 2;
+    int chunks = (int)((target_units + p.rows - 1) / p.rows);
+    const int max_chunks = (V + gran - 1) / gran;
+    if (chunks > max_chunks) chunks = max_chunks;
+    if (chunks < 1) chunks = 1;
+    int per = (V + chunks - 1) / chunks;
+    p.chunk_elems = (per + gran - 1) / gran * gran;
+    p.chunks = (V + p.chunk_elems - 1) / p.chunk_elems;
+    p.off_g = kWsAlign;
+    p.off_pval = align_up(p.off_g + sizeof(int32_t) * (size_t)p.rows, kWsAlign);
+    p.off_pidx = align_up(p.off_pval + sizeof(float) * (size_t)p.rows * p.chunks, kWsAlign);
+    p.total = align_up(p.off_pidx + sizeof(int32_t) * (size_t)p.rows * p.chunks, kWsAlign);
+    return p;
+}
+
+int launch_verify(const int32_t *cand_tok, const void *base_logits, int dtype, int B, int K, int n, int V,
+                  int32_t *accept_len, int32_t *best_cand, int32_t *next_tok, void *ws, const VerifyPlan &plan,
+                  cudaStream_t st) {
+    char *w = (char *)ws;
+    int32_t *err = (int32_t *)w;
+    int32_t *g = (int32_t *)(w + plan.off_g);
+    float *pval = (float *)(w + plan.off_pval);
+    int32_t *pidx = (int32_t *)(w + plan.off_pidx);
+    const long long units = (long long)plan.rows * plan.chunks;
+    const unsigned grid = (unsigned)((units + kWarpsPerBlock - 1) / kWarpsPerBlock);
+    const int esz = dtype == SPEC_BF16 ? 2 : 4;
+    const bool vec = ((uintptr_t)base_logits % 16 == 0) && (V % (16 / esz) == 0);
+    if (dtype == SPEC_BF16) {
+        if (vec) verify_argmax_kernel<true, true><<<grid, kArgmaxThreads, 0, st>>>(base_logits, plan.rows, V, plan.chunk_elems, plan.chunks, pval, pidx);
+        else verify_argmax_kernel<true, false><<<grid, kArgmaxThreads, 0, st>>>(base_logits, plan.rows, V, plan.chunk_elems, plan.chunks, pval, pidx);
+    } else {
+        if (vec) verify_argmax_kernel<false, true><<<grid, kArgmaxThreads, 0, st>>>(base_logits, plan.rows, V, plan.chunk_elems, plan.chunks, pval, pidx);
+        else verify_argmax_kernel<false, false><<<grid, kArgmaxThreads, 0, st>>>(base_logits, plan.rows, V, plan.chunk_elems, plan.chunks, pval, pidx);
+    }
+    SPEC_CUDA_TRY(cudaGetLastError());
+    const size_t smem = sizeof(int32_t) * (size_t)K * (n + 1);
+    verify_accept_kernel<<<B, 128, smem, st>>>(cand_tok, pval, pidx, K, n, plan.chunks, g, accept_len, best_cand,
+                                               next_tok, err);
+    SPEC_CUDA_TRY(cudaGetLastError());
+    return SPEC_OK;
+}
+
+}  // namespace spec

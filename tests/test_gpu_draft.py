@@ -1,0 +1,261 @@
+"""GPU parity of the draft path against the oracle: head logits (tensor-core main loop),
+fused top-k / log-prob epilogue, per-level states and tokens, and whole spec_draft calls."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2404_19124_b200 import synth
+from helpers import LOGIT_TOL, TIE_TOL, DraftChecker, small_cfg, to_oracle_weights, weights_to_cuda, ws_view
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def B():
+    from paper_2404_19124_b200 import build
+    build.build()
+    from paper_2404_19124_b200 import binding
+    return binding
+
+
+def _states(rows, d, seed):
+    g = torch.Generator().manual_seed(seed)
+    return (torch.randn(rows, d, generator=g) * 0.5).to(torch.bfloat16)
+
+
+def _setup(cfg):
+    sw = synth.make_weights(cfg)
+    return sw, to_oracle_weights(sw), weights_to_cuda(sw)
+
+
+# rows: 1 / 4 / 12 are the tiny config's levels; 130 spans two 128-row tiles with a ragged tail;
+# V = 1000 / 1096 leave a ragged last vocabulary tile; d = 200 is not a multiple of the 64-wide K block.
+@pytest.mark.parametrize("impl", [0, 1])
+@pytest.mark.parametrize("rows,V,d", [(1, 1024, 256), (4, 1024, 256), (12, 1024, 256), (130, 1024, 256),
+                                      (33, 1000, 200), (257, 1096, 64), (96, 8000, 512)])
+def test_head_logits_match_oracle(B, impl, rows, V, d):
+    cfg = small_cfg(d_base=d, d_inner=d, V=V, topk=(2, 2), std=None, seed=rows + V)
+    sw, ow, gw = _setup(cfg)
+    h = B.spec_create(gw)
+    B.spec_set_option(h, B.SPEC_OPT_GEMM_IMPL, impl)
+    S = _states(rows, d, 3)
+    got = B.spec_head_logits(h, 1, S.cuda())
+    torch.cuda.synchronize()
+    want = oracle.stage_logits(ow, 1, S.to(torch.float32).numpy())
+    err = np.abs(got.cpu().numpy() - want).max()
+    assert err <= LOGIT_TOL, err
+    assert err <= 2e-3, f"fp32-accumulated logits should be far inside the tolerance, got {err}"
+    B.spec_destroy(h)
+
+
+@pytest.mark.parametrize("block_n", [32, 96, 224, 256])
+def test_head_logits_every_tile_width(B, block_n):
+    cfg = small_cfg(d_base=128, d_inner=320, V=2000, topk=(2, 2), seed=block_n)
+    sw, ow, gw = _setup(cfg)
+    h = B.spec_create(gw)
+    B.spec_set_option(h, B.SPEC_OPT_HEAD_BLOCK_N, block_n)
+    S = _states(140, cfg.d_inner, 9)
+    got = B.spec_head_logits(h, 0, S.cuda())
+    want = oracle.stage_logits(ow, 0, S.to(torch.float32).numpy())
+    assert np.abs(got.cpu().numpy() - want).max() <= 2e-3
+    B.spec_destroy(h)
+
+
+def _check_topk_rows(tok, logp, logits, k):
+    """tok/logp [rows, k] against oracle logits [rows, V] with the tie rule."""
+    tolerated = 0
+    for r in range(logits.shape[0]):
+        ids, vals = oracle.topk(logits[r], k)
+        lse = oracle.logsumexp(logits[r])
+        if np.array_equal(ids, tok[r]):
+            assert np.abs((vals - lse) - logp[r]).max() <= LOGIT_TOL
+            continue
+        tolerated += 1
+        kth = vals[-1]
+        for j in range(k):
+            assert logits[r, tok[r, j]] >= kth - TIE_TOL
+            assert abs((logits[r, tok[r, j]] - lse) - logp[r, j]) <= LOGIT_TOL
+        assert len(set(tok[r].tolist())) == k
+    return tolerated
+
+
+@pytest.mark.parametrize("impl", [0, 1])
+@pytest.mark.parametrize("rows,V,d,k", [(1, 1024, 256, 4), (12, 1024, 256, 2), (130, 1000, 128, 8),
+                                        (40, 8000, 512, 6), (5, 64, 64, 8), (3, 40, 64, 1)])
+def test_head_topk_matches_oracle(B, impl, rows, V, d, k):
+    cfg = small_cfg(d_base=d, d_inner=d, V=V, topk=(2, 2), seed=rows * 7 + k)
+    sw, ow, gw = _setup(cfg)
+    h = B.spec_create(gw)
+    B.spec_set_option(h, B.SPEC_OPT_GEMM_IMPL, impl)
+    S = _states(rows, d, 4)
+    tok, logp, ws = B.spec_head_topk(h, 0, S.cuda(), k)
+    assert B.spec_poll_error(ws) == 0
+    logits = oracle.stage_logits(ow, 0, S.to(torch.float32).numpy())
+    tolerated = _check_topk_rows(tok.cpu().numpy(), logp.cpu().numpy(), logits, k)
+    assert tolerated <= max(1, rows // 20)
+    B.spec_destroy(h)
+
+
+def test_head_topk_exact_ties_prefer_lower_token_id(B):
+    """Duplicate output rows give exactly equal logits: the lower token id must come first,
+    also when the two copies sit in different vocabulary tiles."""
+    cfg = small_cfg(d_base=64, d_inner=64, V=1024, topk=(2, 2), seed=21)
+    sw = synth.make_weights(cfg)
+    for l in range(cfg.n):
+        sw.head[l][700] = sw.head[l][3]
+        sw.head[l][4] = sw.head[l][3]
+    ow, gw = to_oracle_weights(sw), weights_to_cuda(sw)
+    h = B.spec_create(gw)
+    B.spec_set_option(h, B.SPEC_OPT_HEAD_BLOCK_N, 32)
+    # a state aligned with row 3 makes tokens 3, 4 and 700 the tied maximum
+    S = (sw.head[0][3].to(torch.float32) * 40).to(torch.bfloat16)[None].contiguous()
+    tok, logp, _ = B.spec_head_topk(h, 0, S.cuda(), 4)
+    logits = oracle.stage_logits(ow, 0, S.to(torch.float32).numpy())
+    ids, _ = oracle.topk(logits[0], 4)
+    assert ids[:3].tolist() == [3, 4, 700]
+    assert tok.cpu().numpy()[0].tolist() == ids.tolist()
+    B.spec_destroy(h)
+
+
+def _draft_and_check(B, cfg, seqs=None, impl=0, check_levels=False):
+    """Runs spec_draft at the config's full batch and compares the sequences in `seqs`
+    (default: all) with the oracle, one sequence at a time (sequences are independent)."""
+    sw, ow, gw = _setup(cfg)
+    ctx, tok = synth.make_draft_inputs(cfg)
+    h = B.spec_create(gw)
+    B.spec_set_option(h, B.SPEC_OPT_GEMM_IMPL, impl)
+    cand_tok, cand_logp, ws = B.spec_draft(h, ctx.cuda(), tok.cuda(), cfg.topk, cfg.K)
+    assert B.spec_poll_error(ws) == 0
+    ct, lp = cand_tok.cpu().numpy(), cand_logp.cpu().numpy()
+    ctx_bits = synth.bf16_bits(ctx)
+    chk = DraftChecker(ow, cfg.topk, cfg.K)
+    for b in (range(cfg.B) if seqs is None else seqs):
+        chk.check(ctx_bits[b], int(tok[b]), ct[b], lp[b])
+    # the K rows returned are the best K of the library's own leaf scores (property, any size)
+    lay = B.spec_draft_layout(h, cfg.B, cfg.topk, cfg.K)
+    leaf = ws_view(ws, lay.score[cfg.n], cfg.B * cfg.leaves, torch.float32).view(cfg.B, cfg.leaves)
+    top = torch.sort(leaf, dim=1, descending=True, stable=True).values[:, :cfg.K]
+    assert torch.equal(top.cpu(), cand_logp.cpu())
+    if check_levels:
+        o_tok, o_lp, dd = oracle.draft(ow, ctx_bits, tok.numpy(), cfg.topk, cfg.K, dump=True, dump_logits=False)
+        N = cfg.B
+        for l in range(cfg.n if chk.tolerated == 0 else 1):
+            S = ws_view(ws, lay.state[l], N * cfg.d_inner, torch.bfloat16).view(N, cfg.d_inner)
+            S = S.to(torch.float32).cpu().numpy()
+            assert np.allclose(S, dd.states[l], rtol=0.008, atol=2e-4), f"level {l} states"
+            N *= cfg.topk[l]
+            if chk.tolerated == 0:
+                t = ws_view(ws, lay.tok[l + 1], N, torch.int32).cpu().numpy()
+                sc = ws_view(ws, lay.score[l + 1], N, torch.float32).cpu().numpy()
+                assert np.array_equal(t, dd.tok[l]), f"level {l} tokens"
+                assert np.abs(sc - dd.score[l]).max() <= (l + 1) * LOGIT_TOL
+    B.spec_destroy(h)
+    return chk
+
+
+@pytest.mark.parametrize("impl", [0, 1])
+def test_draft_tiny_config(B, impl):
+    chk = _draft_and_check(B, synth.CONFIGS["tiny"], impl=impl, check_levels=True)
+    assert chk.tolerated == 0
+
+
+@pytest.mark.parametrize("topk,K,Bn,V,d_base,d", [((3, 2, 2), 5, 2, 1000, 72, 64), ((1, 1, 1), 1, 3, 512, 64, 64),
+                                                   ((8, 8), 64, 2, 2048, 128, 192), ((2, 2, 2, 2, 2), 7, 5, 640, 64, 128),
+                                                   ((4, 3), 12, 150, 512, 64, 64)])
+def test_draft_odd_shapes(B, topk, K, Bn, V, d_base, d):
+    cfg = small_cfg(d_base=d_base, d_inner=d, V=V, topk=topk, K=K, B=Bn, seed=len(topk) + Bn)
+    chk = _draft_and_check(B, cfg, check_levels=True)
+    assert chk.tolerated <= max(1, Bn // 10)
+
+
+def test_draft_llama2_7b_shape(B):
+    chk = _draft_and_check(B, synth.CONFIGS["llama2-7b"])
+    assert chk.tolerated <= 2
+
+
+@pytest.mark.parametrize("name,seqs", [("llama2-13b", (0, 7, 15)), ("codellama-34b", (0, 31)), ("llama3-8b", (63,))])
+def test_draft_full_size_sampled_sequences(B, name, seqs):
+    """Full batch on the GPU in the benchmark's launch configuration; the oracle re-computes
+    whole trees for a sample of sequences (the full batch would take it minutes to hours)."""
+    _draft_and_check(B, synth.CONFIGS[name], seqs=seqs)
+
+
+def test_draft_is_deterministic_and_stream_ordered(B):
+    cfg = synth.CONFIGS["tiny"]
+    sw, ow, gw = _setup(cfg)
+    ctx, tok = synth.make_draft_inputs(cfg)
+    h = B.spec_create(gw)
+    a = B.spec_draft(h, ctx.cuda(), tok.cuda(), cfg.topk, cfg.K)
+    s = torch.cuda.Stream()
+    s.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(s):
+        b = B.spec_draft(h, ctx.cuda(), tok.cuda(), cfg.topk, cfg.K, stream=s)
+    s.synchronize()
+    torch.cuda.synchronize()
+    assert torch.equal(a[0], b[0]) and torch.equal(a[1], b[1])
+    B.spec_destroy(h)
+
+
+def test_draft_token_out_of_range_sets_error_word_without_trapping(B):
+    cfg = synth.CONFIGS["tiny"]
+    sw, ow, gw = _setup(cfg)
+    ctx, tok = synth.make_draft_inputs(cfg)
+    bad = tok.clone()
+    bad[0] = cfg.V + 5
+    h = B.spec_create(gw)
+    _, _, ws = B.spec_draft(h, ctx.cuda(), bad.cuda(), cfg.topk, cfg.K)
+    assert B.spec_poll_error(ws) == B.SPEC_ERR_TOKEN_RANGE
+    assert B.spec_poll_error(ws) == 0                       # cleared by the poll
+    ct, lp, ws = B.spec_draft(h, ctx.cuda(), tok.cuda(), cfg.topk, cfg.K)   # the context is still usable
+    assert B.spec_poll_error(ws) == 0
+    B.spec_destroy(h)
+
+
+def test_draft_argument_errors(B):
+    cfg = synth.CONFIGS["tiny"]
+    sw, ow, gw = _setup(cfg)
+    ctx, tok = synth.make_draft_inputs(cfg)
+    h = B.spec_create(gw)
+    with pytest.raises(B.SpecError) as e:
+        B.spec_draft(h, ctx.cuda(), tok.cuda(), cfg.topk, cfg.leaves + 1)
+    assert e.value.status == B.SPEC_ERR_SHAPE
+    with pytest.raises(B.SpecError) as e:
+        B.spec_draft(h, ctx.cuda(), tok.cuda(), (9, 1, 1), 2)
+    assert e.value.status == B.SPEC_ERR_SHAPE
+    with pytest.raises(B.SpecError) as e:
+        B.spec_draft(h, ctx.cuda(), tok.cuda(), cfg.topk, cfg.K, workspace=torch.empty(512, dtype=torch.uint8, device="cuda"))
+    assert e.value.status == B.SPEC_ERR_WORKSPACE
+    B.spec_destroy(h)
+
+
+def test_draft_then_verify_chain_and_graph_replay(B):
+    """Draft feeds verify on one stream; a CUDA graph of both replays to the same answer."""
+    cfg = synth.CONFIGS["tiny"]
+    sw, ow, gw = _setup(cfg)
+    ctx, tok = synth.make_draft_inputs(cfg)
+    ctx_d, tok_d = ctx.cuda(), tok.cuda()
+    h = B.spec_create(gw)
+    cand, logp, ws = B.spec_draft(h, ctx_d, tok_d, cfg.topk, cfg.K)
+    logits = synth.make_base_logits(cfg, cand.cpu()).cuda()
+    logits[0, 3, 0, cand[0, 3, 0]] = 30.0
+    logits[0, 3, 1, cand[0, 3, 1]] = 30.0
+    acc, best, nxt, vws = B.spec_verify(cand, logits)
+    torch.cuda.synchronize()
+    o = oracle.verify(cand.cpu().numpy(), synth.bf16_bits(logits), oracle.BF16)
+    assert (acc.item(), best.item(), nxt.item()) == (o[0][0], o[1][0], o[2][0]) and acc.item() >= 2
+    ref = (cand.clone(), logp.clone(), acc.clone(), best.clone(), nxt.clone())
+    s = torch.cuda.Stream()
+    s.wait_stream(torch.cuda.current_stream())
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(s):
+        with torch.cuda.graph(graph, stream=s):
+            B.spec_draft(h, ctx_d, tok_d, cfg.topk, cfg.K, cand_tok=cand, cand_logp=logp, workspace=ws, stream=s)
+            B.spec_verify(cand, logits, accept_len=acc, best_cand=best, next_tok=nxt, workspace=vws, stream=s)
+    for t in (cand, logp, acc, best, nxt):
+        t.zero_()
+    graph.replay()
+    torch.cuda.synchronize()
+    for got, want in zip((cand, logp, acc, best, nxt), ref):
+        assert torch.equal(got, want)
+    B.spec_destroy(h)

@@ -1,0 +1,134 @@
+"""GPU parity of spec_verify against the oracle: bit-exact g, accept_len, best_cand, next_tok."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2404_19124_b200 import synth
+from helpers import ws_view
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def B():
+    from paper_2404_19124_b200 import build
+    build.build()
+    from paper_2404_19124_b200 import binding
+    return binding
+
+
+def _np_logits(x: torch.Tensor):
+    if x.dtype == torch.bfloat16:
+        return synth.bf16_bits(x), oracle.BF16
+    return x.detach().cpu().numpy(), oracle.F32
+
+
+def _run_and_compare(B, cand: torch.Tensor, logits: torch.Tensor):
+    Bn, K, n = cand.shape
+    acc, best, nxt, ws = B.spec_verify(cand.cuda(), logits.cuda())
+    assert B.spec_poll_error(ws) == 0
+    g_gpu = ws_view(ws, 256, Bn * K * (n + 1), torch.int32).cpu().numpy().reshape(Bn, K, n + 1)
+    ln, dt = _np_logits(logits)
+    o_acc, o_best, o_nxt, o_g = oracle.verify(cand.cpu().numpy(), ln, dt, want_g=True)
+    assert np.array_equal(g_gpu, o_g)
+    assert np.array_equal(acc.cpu().numpy(), o_acc)
+    assert np.array_equal(best.cpu().numpy(), o_best)
+    assert np.array_equal(nxt.cpu().numpy(), o_nxt)
+    return o_acc
+
+
+@pytest.mark.parametrize("dtype", [torch.bfloat16, torch.float32])
+@pytest.mark.parametrize("shape", [(1, 8, 3, 1024), (3, 5, 2, 1000), (2, 3, 4, 1021), (2, 7, 1, 8), (1, 1, 1, 1),
+                                   (4, 2, 7, 4100), (2, 64, 4, 50264)])
+def test_verify_small_shapes(B, dtype, shape):
+    Bn, K, n, V = shape
+    g = torch.Generator().manual_seed(sum(shape))
+    logits = (torch.randn(Bn, K, n + 1, V, generator=g) * 2).to(dtype)
+    cand = torch.randint(0, V, (Bn, K, n), generator=g, dtype=torch.int64).to(torch.int32)
+    # plant prefixes of varying length so that accept_len is not always 0
+    am = logits.to(torch.float32).argmax(-1)
+    for b in range(Bn):
+        for k in range(K):
+            m = (b + 2 * k) % (n + 1)
+            cand[b, k, :m] = am[b, k, :m].to(torch.int32)
+    acc = _run_and_compare(B, cand, logits)
+    if K > 1 and n > 1:
+        assert acc.max() > 0
+
+
+def test_verify_unaligned_base_pointer(B):
+    g = torch.Generator().manual_seed(5)
+    V = 1000
+    buf = (torch.randn(2 * 3 * 4 * V + 3, generator=g) * 2).to(torch.bfloat16).cuda()
+    logits = buf[3:].view(2, 3, 4, V)          # 6-byte offset: takes the scalar path
+    assert logits.data_ptr() % 16 != 0
+    cand = torch.randint(0, V, (2, 3, 3), generator=g, dtype=torch.int64).to(torch.int32)
+    acc, best, nxt, ws = B.spec_verify(cand.cuda(), logits)
+    ln = synth.bf16_bits(logits.cpu().contiguous())
+    o = oracle.verify(cand.numpy(), ln, oracle.BF16)
+    assert np.array_equal(acc.cpu().numpy(), o[0]) and np.array_equal(best.cpu().numpy(), o[1])
+    assert np.array_equal(nxt.cpu().numpy(), o[2])
+
+
+def test_verify_ties_nan_and_infinities(B):
+    V = 2048
+    x = torch.zeros(1, 3, 4, V)                           # n = 3; the last row of every candidate is all zeros
+    x[0, 0, 0, [7, 900, 2047]] = 5.0                      # tie: first wins
+    x[0, 0, 1] = float("nan")                             # all NaN -> 0
+    x[0, 0, 2] = float("-inf")                            # all -inf -> 0
+    x[0, 1, 0, 5] = float("nan"); x[0, 1, 0, 1500] = 1.0  # NaN never wins
+    x[0, 1, 1, 100] = float("inf"); x[0, 1, 1, 101] = float("inf")
+    x[0, 1, 2] = -1.0; x[0, 1, 2, 2040] = -0.0            # -0.0 is the maximum
+    x[0, 2, 0] = -3.0; x[0, 2, 0, 1024] = -2.5
+    x[0, 2, 1, 0] = 1.0
+    x[0, 2, 2, V - 1] = 1.0
+    cand = torch.tensor([[[7, 0, 0], [1500, 100, 9], [1024, 0, 5]]], dtype=torch.int32)
+    for dt in (torch.bfloat16, torch.float32):
+        acc = _run_and_compare(B, cand, x.to(dt))
+        assert acc[0] == 3
+
+
+def test_verify_worked_example(B):
+    g = [[2, 3, 0, 4], [2, 3, 1, 0], [2, 0, 0, 3]]
+    x = torch.zeros(1, 3, 4, 5)
+    for k in range(3):
+        for j in range(4):
+            x[0, k, j, g[k][j]] = 10.0
+    cand = torch.tensor([[[2, 4, 1], [2, 3, 0], [1, 0, 0]]], dtype=torch.int32)
+    acc, best, nxt, _ = B.spec_verify(cand.cuda(), x.cuda())
+    assert (acc.item(), best.item(), nxt.item()) == (2, 1, 1)
+    x[0, 1, 1, 1] = 10.0
+    acc, best, nxt, _ = B.spec_verify(cand.cuda(), x.cuda())
+    assert (acc.item(), best.item(), nxt.item()) == (1, 0, 3)
+
+
+@pytest.mark.parametrize("name", ["tiny", "llama2-7b", "llama2-13b", "codellama-34b", "llama3-8b"])
+def test_verify_full_size_configs(B, name):
+    """Full BASELINE shapes in the launch configuration the benchmark times; the oracle
+    checks every row (the CPU arg-max over the whole tensor takes seconds)."""
+    cfg = synth.CONFIGS[name]
+    cand = synth.random_cand_tok(cfg, device="cuda")
+    logits = synth.make_base_logits(cfg, cand, device="cuda")
+    acc, best, nxt, ws = B.spec_verify(cand, logits)
+    torch.cuda.synchronize()
+    rows = cfg.B * cfg.K * (cfg.n + 1)
+    g_gpu = ws_view(ws, 256, rows, torch.int32).cpu().numpy().reshape(cfg.B, cfg.K, cfg.n + 1)
+    bits = synth.bf16_bits(logits)
+    del logits
+    o_acc, o_best, o_nxt, o_g = oracle.verify(cand.cpu().numpy(), bits, oracle.BF16, want_g=True)
+    assert np.array_equal(g_gpu, o_g)
+    assert np.array_equal(acc.cpu().numpy(), o_acc)
+    assert np.array_equal(best.cpu().numpy(), o_best)
+    assert np.array_equal(nxt.cpu().numpy(), o_nxt)
+    if cfg.plant != "none":
+        assert o_acc.max() >= 1
+
+
+def test_verify_argument_errors(B):
+    cand = torch.zeros((1, 2, 2), dtype=torch.int32, device="cuda")
+    logits = torch.zeros((1, 2, 3, 64), dtype=torch.bfloat16, device="cuda")
+    small = torch.empty(256, dtype=torch.uint8, device="cuda")
+    with pytest.raises(B.SpecError) as e:
+        B.spec_verify(cand, logits, workspace=small)
+    assert e.value.status == B.SPEC_ERR_WORKSPACE
