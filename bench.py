@@ -146,6 +146,55 @@ def run_reference(args, cfg):
     print(json.dumps(out), flush=True)
 
 
+def run_only(args, cfg, peaks, dev):
+    """Single-kernel loops (same launch configuration as inside a step) for ncu captures and sweeps."""
+    import torch
+    from paper_2404_19124_b200 import binding as B
+    from paper_2404_19124_b200 import synth
+    stream = torch.cuda.current_stream()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    if args.only == "head":
+        rows = args.rows or cfg.nodes(cfg.n - 1)
+        k = cfg.topk[-1]
+        one = dataclasses.replace(cfg, topk=(k,), K=1)
+        sw = synth.make_weights(one, device=dev)
+        h = B.spec_create(sw)
+        if args.block_n:
+            B.spec_set_option(h, B.SPEC_OPT_HEAD_BLOCK_N, args.block_n)
+        g = torch.Generator(device=dev).manual_seed(5)
+        S = (torch.randn(rows, cfg.d_inner, generator=g, device=dev) * 0.5).to(torch.bfloat16)
+        tok = torch.empty((rows, k), dtype=torch.int32, device=dev)
+        logp = torch.empty((rows, k), dtype=torch.float32, device=dev)
+        ws = torch.empty(B.spec_head_workspace_bytes(h, rows, k), dtype=torch.uint8, device=dev)
+        run = lambda i: B.spec_head_topk(h, 0, S, k, tok=tok, logp=logp, workspace=ws)
+        flops, nbytes = 2.0 * rows * cfg.d_inner * cfg.V, 2.0 * cfg.V * cfg.d_inner + 2.0 * rows * cfg.d_inner
+        what = f"spec_head_topk rows={rows} d_inner={cfg.d_inner} V={cfg.V} topk={k} (GEMM + merge kernels)"
+    else:
+        cand = synth.random_cand_tok(cfg, device=dev)
+        nbytes = cfg.B * cfg.K * (cfg.n + 1) * cfg.V * 2.0
+        n_rot = max(2, min(8, int((512 << 20) // nbytes) + 1))
+        rot = [synth.make_base_logits(dataclasses.replace(cfg, seed=cfg.seed + 100 * i), cand, device=dev)
+               for i in range(n_rot)]
+        vws = torch.empty(B.spec_verify_workspace_bytes(cfg.B, cfg.K, cfg.n, cfg.V, B.SPEC_BF16), dtype=torch.uint8, device=dev)
+        outs = [torch.empty(cfg.B, dtype=torch.int32, device=dev) for _ in range(3)]
+        run = lambda i: B.spec_verify(cand, rot[i % n_rot], accept_len=outs[0], best_cand=outs[1], next_tok=outs[2], workspace=vws)
+        flops = 0.0
+        what = f"spec_verify {cfg.name} logits [{cfg.B},{cfg.K},{cfg.n + 1},{cfg.V}] bf16, {n_rot} rotating buffers"
+    for i in range(args.warmup):
+        run(i)
+    torch.cuda.synchronize()
+    e0.record(stream)
+    for i in range(args.steps):
+        run(i)
+    e1.record(stream)
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / args.steps
+    print(json.dumps({"only": args.only, "what": what, "us": round(ms * 1e3, 2),
+                      "TFLOP/s": round(flops / (ms * 1e-3) / 1e12, 1), "GB/s": round(nbytes / (ms * 1e-3) / 1e9, 1),
+                      "frac_bf16_burst": round(flops / (ms * 1e-3) / 1e12 / peaks["bf16_tflops"], 3),
+                      "frac_hbm": round(nbytes / (ms * 1e-3) / 1e9 / peaks["hbm_gbs"], 3)}), flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -154,6 +203,10 @@ def main():
     ap.add_argument("--config", default="llama2-13b")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--only", default=None, choices=["head", "verify"],
+                    help="kernel-level run for profiling: only the vocabulary-head GEMM (+merge) or only verify")
+    ap.add_argument("--rows", type=int, default=None, help="--only head: rows of the GEMM (default: last level)")
+    ap.add_argument("--block-n", type=int, default=0, help="--only head: force the vocabulary tile width")
     args = ap.parse_args()
 
     from paper_2404_19124_b200 import synth
@@ -183,6 +236,9 @@ def main():
         args.warmup = 3
     peaks = load_peaks()
     dev = f"cuda:{local_rank}"
+    if args.only is not None:
+        run_only(args, cfg, peaks, dev)
+        return
 
     # ---------------------------------------------------------------- inputs, resident in HBM
     sw = synth.make_weights(cfg, device=dev)
