@@ -158,32 +158,124 @@ struct GemmParams {
     int32_t *err;
 };
 
-// ---- epilogue, mode 1: running top-k of one row over the tile + online (max, sum-exp) ----
-struct RowTopK {
-    float v[SPEC_MAX_TOPK];
-    int id[SPEC_MAX_TOPK];
-    __device__ __forceinline__ void reset() {
+// ---- epilogue, mode 1 -----------------------------------------------------------------------
+// One thread owns one accumulator row.  Data-dependent insertion into a sorted list diverges in
+// every warp (each lane inserts at different columns), so the selection is done branch-free:
+//   pass 1  streams the tile once: online (max, sum-exp) and the kCap largest VALUES of the row,
+//           kept sorted by a min/max network (new_v[j] = max(v[j], min(v[j-1], x)));
+//   pass 2  re-reads the tile from TMEM and emits the columns whose value reaches the topk-th
+//           largest; equal values are taken in ascending column order, exactly `topk` entries.
+__device__ __forceinline__ float ex2_approx(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
+template <int kCap>
+__device__ __forceinline__ void epilogue_topk(const GemmParams &p, uint32_t taddr, int row, bool row_ok, int col0,
+                                              int n_tile) {
+    constexpr float kLog2e = 1.4426950408889634f;
+    float best[kCap];
 #pragma unroll
-        for (int j = 0; j < SPEC_MAX_TOPK; ++j) {
-            v[j] = -INFINITY;
-            id[j] = 0x7fffffff;
+    for (int j = 0; j < kCap; ++j) best[j] = -INFINITY;
+    float run_m = -INFINITY, run_s = 0.0f;
+    for (int c = 0; c < p.block_n; c += 32) {
+        float v[32];
+        tmem_ld32(taddr + c, v);
+        const int valid = p.N - (col0 + c);   // columns of this chunk inside the vocabulary
+        if (valid < 32) {
+#pragma unroll
+            for (int i = 0; i < 32; ++i)
+                if (i >= valid) v[i] = -INFINITY;
+        }
+        float cm0 = fmaxf(v[0], v[1]), cm1 = fmaxf(v[2], v[3]);
+#pragma unroll
+        for (int i = 4; i < 32; i += 2) {
+            cm0 = fmaxf(cm0, v[i]);
+            cm1 = fmaxf(cm1, v[i + 1]);
+        }
+        const float cm = fmaxf(cm0, cm1);
+        if (cm > run_m) {
+            run_s *= ex2_approx((run_m - cm) * kLog2e);
+            run_m = cm;
+        }
+        const float ms = run_m * kLog2e;
+        float s0 = 0.0f, s1 = 0.0f, s2 = 0.0f, s3 = 0.0f;
+#pragma unroll
+        for (int i = 0; i < 32; i += 4) {
+            s0 += ex2_approx(fmaf(v[i], kLog2e, -ms));
+            s1 += ex2_approx(fmaf(v[i + 1], kLog2e, -ms));
+            s2 += ex2_approx(fmaf(v[i + 2], kLog2e, -ms));
+            s3 += ex2_approx(fmaf(v[i + 3], kLog2e, -ms));
+        }
+        if (run_m > -INFINITY) run_s += (s0 + s1) + (s2 + s3);
+#pragma unroll
+        for (int i = 0; i < 32; ++i) {
+            const float x = v[i];
+#pragma unroll
+            for (int j = kCap - 1; j > 0; --j) best[j] = fmaxf(best[j], fminf(best[j - 1], x));
+            best[0] = fmaxf(best[0], x);
         }
     }
-    // columns arrive in ascending order, so a strict comparison keeps the lower id among equals
-    __device__ __forceinline__ void push(float x, int col) {
-        if (x > v[SPEC_MAX_TOPK - 1]) {
-            v[SPEC_MAX_TOPK - 1] = x;
-            id[SPEC_MAX_TOPK - 1] = col;
+    // threshold = topk-th largest value of the row in this tile; how many entries lie strictly above it
+    const int topk = p.epi.topk;
+    float thr = best[0];
 #pragma unroll
-            for (int q = SPEC_MAX_TOPK - 1; q > 0; --q) {
-                if (v[q] > v[q - 1]) {
-                    const float fv = v[q]; v[q] = v[q - 1]; v[q - 1] = fv;
-                    const int fi = id[q]; id[q] = id[q - 1]; id[q - 1] = fi;
+    for (int j = 1; j < kCap; ++j)
+        if (j < topk) thr = best[j];
+    int above = 0;
+#pragma unroll
+    for (int j = 0; j < kCap; ++j)
+        if (j < topk && best[j] > thr) ++above;
+    int eq_left = topk - above;
+    const size_t u = (size_t)row * p.n_tiles + n_tile;
+    float *pv = p.epi.part_val + u * SPEC_MAX_TOPK;
+    int32_t *pi = p.epi.part_idx + u * SPEC_MAX_TOPK;
+    int cnt = 0;
+    for (int c = 0; c < p.block_n; c += 32) {
+        float v[32];
+        tmem_ld32(taddr + c, v);
+        const int valid = p.N - (col0 + c);
+        // candidates of this chunk as a bit mask: no per-element branches
+        uint32_t mask = 0;
+#pragma unroll
+        for (int i = 0; i < 32; ++i) mask |= (v[i] >= thr ? 1u : 0u) << i;
+        if (valid < 32) mask &= valid > 0 ? ((1u << valid) - 1u) : 0u;
+        if (!row_ok) mask = 0;
+        while (mask) {   // ascending columns; a handful of iterations per tile
+            const int bpos = __ffs(mask) - 1;
+            mask &= mask - 1;
+            // x = v[bpos] through a select tree (bpos is data dependent, v lives in registers)
+            float t16[16], t8[8], t4[4], t2[2];
+#pragma unroll
+            for (int i = 0; i < 16; ++i) t16[i] = (bpos & 1) ? v[2 * i + 1] : v[2 * i];
+#pragma unroll
+            for (int i = 0; i < 8; ++i) t8[i] = (bpos & 2) ? t16[2 * i + 1] : t16[2 * i];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) t4[i] = (bpos & 4) ? t8[2 * i + 1] : t8[2 * i];
+#pragma unroll
+            for (int i = 0; i < 2; ++i) t2[i] = (bpos & 8) ? t4[2 * i + 1] : t4[2 * i];
+            const float x = (bpos & 16) ? t2[1] : t2[0];
+            const bool gt = x > thr;
+            if (gt || eq_left > 0) {
+                if (!gt) --eq_left;
+                if (cnt < topk) {
+                    pv[cnt] = x;
+                    pi[cnt] = col0 + c + bpos;
                 }
+                ++cnt;
             }
         }
     }
-};
+    if (row_ok) {
+        for (; cnt < topk; ++cnt) {   // fewer than topk comparable values (NaN rows, tiny tiles)
+            pv[cnt] = -INFINITY;
+            pi[cnt] = 0x7fffffff;
+        }
+        p.epi.part_ms[2 * u] = run_m;
+        p.epi.part_ms[2 * u + 1] = run_s;
+    }
+}
 
 __global__ void __launch_bounds__(kThreads, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
@@ -316,50 +408,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
                     }
                 }
             } else {
-                RowTopK tk;
-                tk.reset();
-                float run_m = -INFINITY, run_s = 0.0f;
-                constexpr float kLog2e = 1.4426950408889634f;
-                for (int c = 0; c < p.block_n; c += 32) {
-                    float v[32];
-                    tmem_ld32(taddr + c, v);
-                    const int valid = p.N - (col0 + c);   // columns of this chunk inside the vocabulary
-                    if (row_ok && valid > 0) {
-                        float cm = -INFINITY;
-#pragma unroll
-                        for (int i = 0; i < 32; ++i) {
-                            if (i >= valid) v[i] = -INFINITY;
-                            cm = fmaxf(cm, v[i]);
-                        }
-                        if (cm > run_m) {
-                            run_s *= exp2f((run_m - cm) * kLog2e);
-                            run_m = cm;
-                        }
-                        const float ms = run_m * kLog2e;
-                        float s = 0.0f;
-#pragma unroll
-                        for (int i = 0; i < 32; ++i) s += exp2f(fmaf(v[i], kLog2e, -ms));
-                        run_s += s;
-                        if (cm > tk.v[SPEC_MAX_TOPK - 1]) {
-#pragma unroll
-                            for (int i = 0; i < 32; ++i) tk.push(v[i], col0 + c + i);
-                        }
-                    }
-                }
-                if (row_ok) {
-                    const size_t u = (size_t)row * p.n_tiles + n_tile;
-                    float *pv = p.epi.part_val + u * SPEC_MAX_TOPK;
-                    int32_t *pi = p.epi.part_idx + u * SPEC_MAX_TOPK;
-#pragma unroll
-                    for (int j = 0; j < SPEC_MAX_TOPK; ++j) {
-                        if (j < p.epi.topk) {
-                            pv[j] = tk.v[j];
-                            pi[j] = tk.id[j];
-                        }
-                    }
-                    p.epi.part_ms[2 * u] = run_m;
-                    p.epi.part_ms[2 * u + 1] = run_s;
-                }
+                if (p.epi.topk <= 4) epilogue_topk<4>(p, taddr, row, row_ok, col0, n_tile);
+                else epilogue_topk<SPEC_MAX_TOPK>(p, taddr, row, row_ok, col0, n_tile);
             }
             tc_fence_before();
             __syncwarp();
