@@ -19,7 +19,25 @@ import numpy as np
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
 _SRC = os.path.join(_HERE, "spec_oracle.c")
-_LIB = os.path.join(_HERE, "libspec_oracle.so")
+
+
+def _cpu_tag() -> str:
+    """Short hash of this host's CPU feature flags: the library is compiled with -march=native, so a
+    copy built on another machine must not be loaded here."""
+    import hashlib
+    flags = ""
+    try:
+        with open("/proc/cpuinfo") as f:
+            for line in f:
+                if line.startswith("flags"):
+                    flags = line
+                    break
+    except OSError:
+        pass
+    return hashlib.sha1(flags.encode()).hexdigest()[:10]
+
+
+_LIB = os.path.join(_HERE, f"libspec_oracle.{_cpu_tag()}.so")
 
 MAX_HEADS = 8
 BF16, F32 = 0, 1
