@@ -224,6 +224,7 @@ def main():
 
     import torch
     from paper_2404_19124_b200 import binding as B
+    from paper_2404_19124_b200 import shard
 
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device: the draft/verify path has no CPU fallback")
@@ -272,11 +273,7 @@ def main():
         torch.cuda.synchronize()
 
     def max_over_ranks(x: float) -> float:
-        if dist is None:
-            return x
-        t = torch.tensor([x], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        return float(t.item())
+        return shard.max_over_ranks(x, dist, dev)
 
     # ---------------------------------------------------------------- device-resident timing
     for i in range(args.warmup):
@@ -403,7 +400,7 @@ def main():
 
     launches_per_step = 4 * n + 1 + 2
     out = {
-        "metric": METRIC, "value": world * Bn / (ms_step * 1e-3), "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "metric": METRIC, "value": shard.whole_job_rate(Bn, world, ms_step * 1e-3), "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
         "config": {"workload": cfg.name, "B": Bn, "K": K, "n_heads": n, "topk": list(cfg.topk), "V": V,
@@ -412,7 +409,7 @@ def main():
                    "parallelism": f"replicas x{world}, sequences independent, no collective"},
         "roofline": roof, "roofline_verify": roof_verify, "head_gemms": head_hbm, "kernel_us": kernels,
         "cpu_baseline": cpu,
-        "e2e": {"value": world * Bn / (e2e_ms * 1e-3), "unit": UNIT, "ms_per_step": e2e_ms,
+        "e2e": {"value": shard.whole_job_rate(Bn, world, e2e_ms * 1e-3), "unit": UNIT, "ms_per_step": e2e_ms,
                 "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
         "gpu_launches": launches_per_step * args.steps,
         "clocks": clocks, "synthetic_tokens_per_step": tau,
