@@ -2,9 +2,11 @@
 // i.e. K-major for both), fp32 accumulation in tensor memory (TMEM).
 //
 // It serves the two contractions of a speculator stage (Sec. 3.1 of arXiv 2404.19124): the
-// projection of the parent states (epilogue mode 0: fp32 store) and the vocabulary head
-// (epilogue mode 1: the logits tile stays on the SM; each accumulator row is reduced to a
-// partial top-k list and a (max, sum-exp) pair, so full logits never reach HBM).
+// projection of the parent states (epilogue mode 0: fp32 store; mode 2: the operands are swapped
+// so that the weight matrix fills the 128-row side of the MMA when there are few states, the
+// contraction is split over several CTAs and every split stores its partial result transposed)
+// and the vocabulary head (epilogue mode 1: the logits tile stays on the SM; each accumulator row
+// is reduced to a partial top-k list and a (max, sum-exp) pair, so full logits never reach HBM).
 //
 // Structure: persistent CTAs, one per SM, static round-robin over (n_tile, m_tile) tiles with
 // the m index fastest, so the CTAs that share a weight tile run at the same time and the
@@ -30,8 +32,8 @@ constexpr int kBlockM = 128;
 constexpr int kBlockK = 64;            // 64 bf16 = 128 bytes = one swizzle span
 constexpr int kUmmaK = 16;
 constexpr int kThreads = 192;
-constexpr int kMaxStages = 8;
-constexpr int kSmemLimit = 227 * 1024;
+constexpr int kMaxStages = 12;
+constexpr int kSmemLimit = 222 * 1024;   // leaves room on the SM for the small kernels that overlap with this one
 constexpr uint32_t kSpinFast = 1u << 14;
 constexpr uint32_t kSpinMax = 1u << 24;
 
@@ -153,6 +155,7 @@ struct GemmParams {
     int M, N, Kd;
     int block_n, stages, tmem_cols;
     int m_tiles, n_tiles;
+    int splits, kb_per_split;   // split-K: tile = (m_tile, n_tile, split), split slowest
     uint32_t stage_bytes, a_bytes;
     GemmEpilogue epi;
     int32_t *err;
@@ -287,7 +290,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int num_kb = (p.Kd + kBlockK - 1) / kBlockK;
-    const int num_tiles = p.m_tiles * p.n_tiles;
+    const int mn_tiles = p.m_tiles * p.n_tiles;
+    const int num_tiles = mn_tiles * p.splits;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < p.stages; ++s) {
@@ -313,22 +317,47 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
     tc_fence_after();
     const uint32_t tmem_base = bars->tmem_base;
 
+    griddep_launch();   // the next kernel in the stream may start its own set-up now
     if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer
         if (lane == 0) {
+            // Which operand holds the weights (written by no kernel) and which the states (written by
+            // the preceding kernel): the first fill of the ring fetches weights only, then waits for
+            // the preceding grid, then adds the states.
+            const bool w_is_a = p.epi.mode == 2;
+            int n_pre = 0;
+            if ((int)blockIdx.x < num_tiles) {
+                const int tile = blockIdx.x;
+                const int split = tile / mn_tiles, mn = tile - split * mn_tiles;
+                const int m_tile = mn % p.m_tiles, n_tile = mn / p.m_tiles;
+                const int kb0 = split * p.kb_per_split, kb1 = min(num_kb, kb0 + p.kb_per_split);
+                n_pre = min(p.stages, kb1 - kb0);
+                for (int i = 0; i < n_pre; ++i) {
+                    uint8_t *sa = tiles + (size_t)i * p.stage_bytes;
+                    mbar_arrive_expect_tx(&bars->full[i], p.stage_bytes);
+                    if (w_is_a) tma_load_2d(sa, &tmap_a, (kb0 + i) * kBlockK, m_tile * kBlockM, &bars->full[i]);
+                    else tma_load_2d(sa + p.a_bytes, &tmap_b, (kb0 + i) * kBlockK, n_tile * p.block_n, &bars->full[i]);
+                }
+            }
+            griddep_wait();
             int stage = 0;
             uint32_t phase = 0;
-            int issued = 0;   // loads issued and not known to be consumed, for the abort path
+            int issued = 0;   // k blocks issued so far; also bounds the abort path's wait for copies in flight
             bool ok = true;
             for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x) {
-                const int m_tile = tile % p.m_tiles, n_tile = tile / p.m_tiles;
-                for (int kb = 0; kb < num_kb; ++kb) {
-                    if (!mbar_wait(&bars->empty[stage], phase ^ 1u, bars, p.err)) { ok = false; break; }
+                const int split = tile / mn_tiles, mn = tile - split * mn_tiles;
+                const int m_tile = mn % p.m_tiles, n_tile = mn / p.m_tiles;
+                const int kb0 = split * p.kb_per_split, kb1 = min(num_kb, kb0 + p.kb_per_split);
+                for (int kb = kb0; kb < kb1; ++kb) {
                     uint8_t *sa = tiles + (size_t)stage * p.stage_bytes;
                     uint8_t *sb = sa + p.a_bytes;
-                    mbar_arrive_expect_tx(&bars->full[stage], p.stage_bytes);
-                    tma_load_2d(sa, &tmap_a, kb * kBlockK, m_tile * kBlockM, &bars->full[stage]);
-                    tma_load_2d(sb, &tmap_b, kb * kBlockK, n_tile * p.block_n, &bars->full[stage]);
+                    const bool prefetched = issued < n_pre;   // weights of this stage are already on their way
+                    if (!prefetched) {
+                        if (!mbar_wait(&bars->empty[stage], phase ^ 1u, bars, p.err)) { ok = false; break; }
+                        mbar_arrive_expect_tx(&bars->full[stage], p.stage_bytes);
+                    }
+                    if (!prefetched || !w_is_a) tma_load_2d(sa, &tmap_a, kb * kBlockK, m_tile * kBlockM, &bars->full[stage]);
+                    if (!prefetched || w_is_a) tma_load_2d(sb, &tmap_b, kb * kBlockK, n_tile * p.block_n, &bars->full[stage]);
                     ++issued;
                     if (++stage == p.stages) { stage = 0; phase ^= 1u; }
                 }
@@ -343,9 +372,12 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
                     for (uint32_t it = 0; it < (1u << 20) && !mbar_try_wait(&bars->full[s], ph); ++it) __nanosleep(32);
                 }
             }
+        } else {
+            griddep_wait();
         }
     } else if (warp == 1) {
         // ------------------------------------------------------------------ MMA issuer
+        griddep_wait();
         if (lane == 0) {
             const uint32_t idesc = make_instr_desc(kBlockM, p.block_n);
             int stage = 0, acc = 0;
@@ -355,7 +387,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
                 if (!mbar_wait(&bars->acc_empty[acc], acc_phase ^ 1u, bars, p.err)) { ok = false; break; }
                 tc_fence_after();
                 const uint32_t tmem_d = tmem_base + (uint32_t)(acc * p.block_n);
-                for (int kb = 0; kb < num_kb; ++kb) {
+                const int split = tile / mn_tiles;
+                const int kb0 = split * p.kb_per_split, kb1 = min(num_kb, kb0 + p.kb_per_split);
+                for (int kb = kb0; kb < kb1; ++kb) {
                     if (!mbar_wait(&bars->full[stage], phase, bars, p.err)) { ok = false; break; }
                     tc_fence_after();
                     const uint32_t sa = smem_u32(tiles + (size_t)stage * p.stage_bytes);
@@ -364,7 +398,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
                     for (int k = 0; k < kBlockK / kUmmaK; ++k) {
                         const uint64_t adesc = make_smem_desc(sa + k * kUmmaK * 2);
                         const uint64_t bdesc = make_smem_desc(sb + k * kUmmaK * 2);
-                        umma_bf16(tmem_d, adesc, bdesc, idesc, (kb | k) != 0 ? 1u : 0u);
+                        umma_bf16(tmem_d, adesc, bdesc, idesc, ((kb - kb0) | k) != 0 ? 1u : 0u);
                     }
                     umma_commit(&bars->empty[stage]);   // frees the stage once these MMAs have read it
                     if (++stage == p.stages) { stage = 0; phase ^= 1u; }
@@ -376,13 +410,15 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
         }
     } else {
         // ------------------------------------------------------------------ epilogue warps
+        griddep_wait();
         const int quarter = warp & 3;               // TMEM lane quarter this warp may read
         const int row_in_tile = quarter * 32 + lane;
         int acc = 0;
         uint32_t acc_phase = 0;
         bool ok = true;
         for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x) {
-            const int m_tile = tile % p.m_tiles, n_tile = tile / p.m_tiles;
+            const int split = tile / mn_tiles, mn = tile - split * mn_tiles;
+            const int m_tile = mn % p.m_tiles, n_tile = mn / p.m_tiles;
             if (!mbar_wait(&bars->acc_full[acc], acc_phase, bars, p.err)) { ok = false; break; }
             tc_fence_after();
             const int row = m_tile * kBlockM + row_in_tile;
@@ -405,6 +441,20 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
                             for (int i = 0; i < 32; ++i)
                                 if (i < valid) dst[i] = v[i];
                         }
+                    }
+                }
+            } else if (p.epi.mode == 2) {
+                // transposed store of one split-K partial: out[split][col][row]; a warp's 32 rows are
+                // consecutive addresses, so every store instruction is one 128-byte line
+                float *dst0 = p.epi.out + (size_t)split * p.epi.split_stride + row;
+                for (int c = 0; c < p.block_n; c += 32) {
+                    float v[32];
+                    tmem_ld32(taddr + c, v);
+                    if (row_ok) {
+                        const int valid = p.N - (col0 + c);
+#pragma unroll
+                        for (int i = 0; i < 32; ++i)
+                            if (i < valid) dst0[(size_t)(col0 + c + i) * p.epi.ldc] = v[i];
                     }
                 }
             } else {
@@ -518,6 +568,10 @@ int launch_gemm_tc(const void *A, const void *B, int M, int N, int Kd, int block
     p.n_tiles = (N + block_n - 1) / block_n;
     p.epi = epi;
     p.err = err;
+    const int num_kb = (Kd + kBlockK - 1) / kBlockK;
+    p.splits = epi.mode == 2 && epi.splits > 1 ? epi.splits : 1;
+    p.kb_per_split = (num_kb + p.splits - 1) / p.splits;
+    if ((p.splits - 1) * p.kb_per_split >= num_kb) return SPEC_ERR_SHAPE;   // every split must own a K block
 
     const size_t smem = 1024 + (size_t)p.stages * p.stage_bytes + sizeof(Barriers);
     static bool attr_set[64] = {};
@@ -527,10 +581,9 @@ int launch_gemm_tc(const void *A, const void *B, int M, int N, int Kd, int block
         SPEC_CUDA_TRY(cudaFuncSetAttribute(gemm_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemLimit));
         if (dev >= 0 && dev < 64) attr_set[dev] = true;
     }
-    const long long tiles = (long long)p.m_tiles * p.n_tiles;
+    const long long tiles = (long long)p.m_tiles * p.n_tiles * p.splits;
     const int grid = (int)(tiles < num_sms() ? tiles : num_sms());
-    gemm_tc_kernel<<<grid, kThreads, smem, st>>>(ta, tb, p);
-    SPEC_CUDA_TRY(cudaGetLastError());
+    SPEC_CUDA_TRY(launch_pdl(gemm_tc_kernel, dim3(grid), dim3(kThreads), smem, st, ta, tb, p));
     return SPEC_OK;
 }
 

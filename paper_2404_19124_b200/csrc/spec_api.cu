@@ -52,6 +52,7 @@ struct DraftPlan {
     int L;
     spec_draft_layout_t lay;
     int proj_block_n[SPEC_MAX_HEADS];
+    int proj_splits[SPEC_MAX_HEADS];   // > 0: swapped split-K projection (few parent rows); 0: plain
 };
 
 int head_block_n_for(const spec_handle_s *h, int rows) {
@@ -62,6 +63,20 @@ int head_block_n_for(const spec_handle_s *h, int rows) {
 int proj_block_n_for(const spec_handle_s *h, int rows) {
     if (h->proj_block_n > 0) return h->proj_block_n;
     return choose_block_n(rows, h->w.d_inner, num_sms(), rows > 128);
+}
+
+// Projection with at most 128 parent rows: the weight matrix takes the 128-row side of the MMA,
+// the states the narrow side, and the contraction is cut into as many K ranges as keep every SM
+// busy (each range at least four 64-wide K blocks).  Returns 0 when the plain form is used.
+int proj_splits_for(const spec_handle_s *h, int parent_rows, int d_in) {
+    if (h->gemm_impl != 0 || parent_rows > 128 || h->proj_block_n > 0) return 0;
+    const int m_tiles = (h->w.d_inner + 127) / 128, num_kb = (d_in + 63) / 64;
+    int splits = num_sms() / m_tiles;
+    if (splits > num_kb / 4) splits = num_kb / 4;
+    if (splits > 8) splits = 8;
+    if (splits < 1) splits = 1;
+    const int per = (num_kb + splits - 1) / splits;
+    return (num_kb + per - 1) / per;   // no empty range
 }
 
 int make_draft_plan(const spec_handle_s *h, int B, const int32_t *topk, int K, DraftPlan *p) {
@@ -91,23 +106,26 @@ int make_draft_plan(const spec_handle_s *h, int B, const int32_t *topk, int K, D
         y.score[l] = off;
         off = align_up(off + sizeof(float) * (size_t)p->N[l], kWsAlign);
     }
-    int max_parent_rows = B;
+    size_t max_proj_floats = 0;
     size_t max_part_units = 0;
     int max_rows = 0;
     for (int l = 0; l < p->n; ++l) {
         y.state[l] = off;
         off = align_up(off + 2 * (size_t)p->N[l] * w.d_inner, kWsAlign);
-        if (l > 0 && p->N[l - 1] > max_parent_rows) max_parent_rows = p->N[l - 1];
+        const int parent_rows = l == 0 ? B : p->N[l - 1];
+        p->proj_splits[l] = proj_splits_for(h, parent_rows, d_in_of(w, l));
+        const size_t pf = (size_t)(p->proj_splits[l] > 0 ? p->proj_splits[l] : 1) * parent_rows * w.d_inner;
+        if (pf > max_proj_floats) max_proj_floats = pf;
         const int bn = head_block_n_for(h, p->N[l]);
         y.block_n[l] = bn;
         y.n_tiles[l] = (w.V + bn - 1) / bn;
         const size_t units = (size_t)p->N[l] * y.n_tiles[l];
         if (units > max_part_units) max_part_units = units;
         if (p->N[l] > max_rows) max_rows = p->N[l];
-        p->proj_block_n[l] = proj_block_n_for(h, l == 0 ? B : p->N[l - 1]);
+        p->proj_block_n[l] = proj_block_n_for(h, parent_rows);
     }
     y.proj = off;
-    off = align_up(off + sizeof(float) * (size_t)max_parent_rows * w.d_inner, kWsAlign);
+    off = align_up(off + sizeof(float) * max_proj_floats, kWsAlign);
     y.part_val = off;
     off = align_up(off + sizeof(float) * max_part_units * SPEC_MAX_TOPK, kWsAlign);
     y.part_idx = off;
@@ -304,13 +322,27 @@ int spec_draft(spec_handle_t h, const void *ctx_state, const int32_t *last_tok, 
         const float *score_l = l == 0 ? nullptr : (const float *)(ws + p.lay.score[l]);
         void *S = ws + p.lay.state[l];
         // projection of every distinct parent state: P = S_parent * Wp^T
-        rc = run_gemm_store(h, parent_states, w.proj[l], parent_rows, w.d_inner, d_in_of(w, l), p.proj_block_n[l], P,
-                            err, st);
+        const int splits = p.proj_splits[l];
+        const size_t split_stride = (size_t)parent_rows * w.d_inner;
+        if (splits > 0) {
+            GemmEpilogue e{};
+            e.mode = 2;
+            e.out = P;
+            e.ldc = w.d_inner;
+            e.splits = splits;
+            e.split_stride = split_stride;
+            rc = launch_gemm_tc(w.proj[l], parent_states, w.d_inner, parent_rows, d_in_of(w, l),
+                                (parent_rows + 31) / 32 * 32, e, err, st);
+        } else {
+            rc = run_gemm_store(h, parent_states, w.proj[l], parent_rows, w.d_inner, d_in_of(w, l),
+                                p.proj_block_n[l], P, err, st);
+        }
         if (rc != SPEC_OK) return rc;
         SPEC_PROF_MARK();
         // gather + mix + LayerNorm + GELU -> bf16 state of every node of this level
-        rc = launch_mix_ln_gelu(P, w.emb[l], tok_l, w.ln_gamma[l], w.ln_beta[l], rows, w.d_inner, w.V,
-                                l == 0 ? 1 : topk[l - 1], w.state_weight, w.emb_weight, w.ln_eps, S, err, st);
+        rc = launch_mix_ln_gelu(P, splits > 0 ? splits : 1, split_stride, w.emb[l], tok_l, w.ln_gamma[l],
+                                w.ln_beta[l], rows, w.d_inner, w.V, l == 0 ? 1 : topk[l - 1], w.state_weight,
+                                w.emb_weight, w.ln_eps, S, err, st);
         if (rc != SPEC_OK) return rc;
         SPEC_PROF_MARK();
         // vocabulary head with the fused per-tile top-k / log-sum-exp epilogue

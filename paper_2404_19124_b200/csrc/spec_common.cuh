@@ -27,9 +27,36 @@ __device__ __forceinline__ uint32_t float_to_bf16_bits(float f) {
     return u >> 16;
 }
 
+// Programmatic dependent launch: every kernel of the library is enqueued with the
+// "programmatic stream serialization" attribute.  A kernel lets its successor start early
+// (griddep_launch, executed by all threads near the top) so the successor's launch latency,
+// set-up and loads of data that no kernel writes (the weights) overlap this kernel's tail;
+// nothing that an earlier kernel produces is touched before griddep_wait, which returns once
+// the preceding grid has completed and its writes are visible.  Every thread of every kernel
+// executes griddep_wait, so "grid N complete" implies "grid N-1 complete" along the whole chain.
+__device__ __forceinline__ void griddep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void griddep_launch() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
 // Host-side bookkeeping ------------------------------------------------------------------
 void set_last_cuda_error(int e);
 int num_sms();
+
+// cudaLaunchKernelEx with the programmatic-serialization attribute set.
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st,
+                              Args... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
+}
 
 #define SPEC_CUDA_TRY(expr)                              \
     do {                                                 \
@@ -43,8 +70,11 @@ int num_sms();
 // ---- verify (verify_kernels.cu) ----------------------------------------------------------
 struct VerifyPlan {
     int rows;          // B * K * (n + 1)
-    int chunk_elems;   // elements of one (row, chunk) work unit
-    int chunks;        // chunks per row
+    int chunk_elems;   // scalar fallback: elements of one (row, chunk) work unit
+    int chunks;        // scalar fallback: chunks per row
+    int vpr;           // streamed form: 16-byte vectors per row (0 when rows are not whole vectors)
+    int vec_per_warp;  // streamed form: vectors in one warp's contiguous range
+    int slots;         // partial slots reserved per row
     size_t off_g;      // int32 [rows]
     size_t off_pval;   // fp32 [rows, chunks]
     size_t off_pidx;   // int32 [rows, chunks]
@@ -58,9 +88,12 @@ int launch_verify(const int32_t *cand_tok, const void *base_logits, int dtype, i
 // ---- tensor-core GEMM (gemm_tcgen05.cu) -------------------------------------------------
 // C[M, N] = A[M, Kd] * B[N, Kd]^T, A and B bf16 row-major (K-major), fp32 accumulation in TMEM.
 struct GemmEpilogue {
-    int mode;          // 0: store fp32 C; 1: per-row partial top-k + (max, sum-exp) per tile
-    float *out;        // mode 0: [M, N] row-major
-    int ldc;           // mode 0: leading dimension of out
+    int mode;          // 0: store fp32 C; 1: per-row partial top-k + (max, sum-exp) per tile;
+                       // 2: split-K partials stored transposed, out[split][n][m]
+    float *out;        // mode 0: [M, N] row-major; mode 2: [splits][N][ldc]
+    int ldc;           // mode 0 / 2: leading dimension of out
+    int splits;        // mode 2: number of K ranges, each handled by its own tile
+    size_t split_stride; // mode 2: elements between the partial results of consecutive splits
     float *part_val;   // mode 1: [M, n_tiles, SPEC_MAX_TOPK]
     int32_t *part_idx; // mode 1: [M, n_tiles, SPEC_MAX_TOPK]
     float *part_ms;    // mode 1: [M, n_tiles, 2]
@@ -77,9 +110,10 @@ int launch_partials_from_logits(const float *logits, int M, int N, int block_n, 
                                 int32_t *part_idx, float *part_ms, cudaStream_t st);
 
 // ---- row kernels of the draft (draft_kernels.cu) ----------------------------------------
-int launch_mix_ln_gelu(const float *P, const void *emb, const int32_t *tok, const float *gamma, const float *beta,
-                       int rows, int d_inner, int V, int parent_div, float a, float b, float eps, void *S_out,
-                       int32_t *err, cudaStream_t st);
+// P: `p_splits` partial projections, `p_split_stride` floats apart, summed on load.
+int launch_mix_ln_gelu(const float *P, int p_splits, size_t p_split_stride, const void *emb, const int32_t *tok,
+                       const float *gamma, const float *beta, int rows, int d_inner, int V, int parent_div, float a,
+                       float b, float eps, void *S_out, int32_t *err, cudaStream_t st);
 int launch_merge_expand(const float *part_val, const int32_t *part_idx, const float *part_ms, int rows, int n_tiles,
                         int topk, const float *score_in, int32_t *tok_out, float *score_out, int score_is_logp,
                         cudaStream_t st);

@@ -2,11 +2,15 @@
 // a bandwidth-bound streaming arg-max over every row of the base model's logits followed by
 // the longest-matching-prefix / best-candidate reduction.
 //
-// Kernel 1 (verify_argmax_kernel): the B*K*(n+1) rows are cut into (row, chunk) work units,
-//   one warp per unit, 128-bit streaming loads with four loads in flight per lane.  For bf16
-//   the running maximum is taken on packed pairs (max.bf16x2), the element index is only
-//   resolved when a vector beats the lane's current best, so the common case costs about one
-//   ALU operation per element.  Each unit writes one (value, index) partial.
+// Kernel 1 (verify_stream_kernel): the whole tensor is one run of 16-byte vectors, cut into equal
+//   contiguous ranges, one per warp, sized so that the grid is a single wave of resident CTAs on
+//   every SM (no ragged second wave).  A warp walks the row segments inside its range with eight
+//   128-bit streaming loads in flight per lane.  For bf16 the running maximum is taken on packed
+//   pairs (max.bf16x2) and the element index is only resolved when a vector beats the lane's
+//   current best, so the common case costs about one ALU operation per element.  Each (row, warp)
+//   intersection writes one (value, index) partial into the row's slot list.
+//   (verify_argmax_kernel is the scalar fallback for unaligned tensors or odd row lengths: fixed
+//   chunks per row, one warp per chunk.)
 // Kernel 2 (verify_accept_kernel): one CTA per sequence folds the partials of its K*(n+1)
 //   rows into g[b,k,j], counts the matching prefix of every candidate and picks the best one.
 #include <float.h>
@@ -76,10 +80,61 @@ __device__ __forceinline__ void warp_argmax(float &best, int &idx) {
     }
 }
 
+constexpr int kStreamUnroll = 8;
+
+// vec_per_warp vectors per warp; row r owns vectors [r * vpr, (r + 1) * vpr); the partial of the
+// (row, warp) intersection goes to slot  warp - first_warp(row)  of the row.
+template <bool kBf16>
+__global__ void __launch_bounds__(kArgmaxThreads, 4)
+verify_stream_kernel(const uint4 *__restrict__ logits, long long total_vec, int vpr, int vec_per_warp, int slots,
+                     float *__restrict__ pval, int32_t *__restrict__ pidx) {
+    griddep_launch();
+    griddep_wait();
+    constexpr int kEpv = kBf16 ? 8 : 4;
+    const int lane = threadIdx.x & 31;
+    const long long w = (long long)blockIdx.x * kWarpsPerBlock + (threadIdx.x >> 5);
+    const long long beg = w * vec_per_warp;
+    if (beg >= total_vec) return;
+    const long long end = min(total_vec, beg + vec_per_warp);
+    long long sb = beg;
+    int row = (int)(beg / vpr);
+    while (sb < end) {
+        const long long row0 = (long long)row * vpr;
+        const long long se = min(end, row0 + vpr);   // end of this row's segment inside the range
+        float best = -INFINITY;
+        int idx = kIdxNone;
+        for (long long p0 = sb + lane; p0 < se; p0 += 32 * kStreamUnroll) {
+            uint4 q[kStreamUnroll];
+#pragma unroll
+            for (int u = 0; u < kStreamUnroll; ++u)
+                if (p0 + 32 * u < se) q[u] = ld_stream(logits + p0 + 32 * u);
+#pragma unroll
+            for (int u = 0; u < kStreamUnroll; ++u) {
+                if (p0 + 32 * u < se) {
+                    const int base = (int)(p0 + 32 * u - row0) * kEpv;
+                    if (kBf16) consume_bf16(q[u], base, best, idx);
+                    else consume_f32(q[u], base, best, idx);
+                }
+            }
+        }
+        warp_argmax(best, idx);
+        if (lane == 0) {
+            const long long first_w = row0 / vec_per_warp;
+            const size_t slot = (size_t)row * slots + (size_t)(w - first_w);
+            pval[slot] = best;
+            pidx[slot] = idx;
+        }
+        sb = se;
+        ++row;
+    }
+}
+
 template <bool kBf16, bool kVector>
 __global__ void __launch_bounds__(kArgmaxThreads)
 verify_argmax_kernel(const void *__restrict__ logits, int rows, int V, int chunk_elems, int chunks,
                      float *__restrict__ pval, int32_t *__restrict__ pidx) {
+    griddep_launch();
+    griddep_wait();
     const int lane = threadIdx.x & 31;
     const long long unit = (long long)blockIdx.x * kWarpsPerBlock + (threadIdx.x >> 5);
     if (unit >= (long long)rows * chunks) return;
@@ -127,18 +182,26 @@ verify_argmax_kernel(const void *__restrict__ logits, int rows, int V, int chunk
 
 __global__ void __launch_bounds__(128)
 verify_accept_kernel(const int32_t *__restrict__ cand_tok, const float *__restrict__ pval,
-                     const int32_t *__restrict__ pidx, int K, int n, int chunks, int32_t *__restrict__ g_out,
+                     const int32_t *__restrict__ pidx, int K, int n, int slots, int vpr, int vec_per_warp,
+                     int32_t *__restrict__ g_out,
                      int32_t *__restrict__ accept_len, int32_t *__restrict__ best_cand,
                      int32_t *__restrict__ next_tok, int32_t *err) {
     extern __shared__ int32_t g_s[];   // [K * (n + 1)]
     __shared__ unsigned int key_s;
     const int b = blockIdx.x, rows_b = K * (n + 1);
+    griddep_launch();
+    griddep_wait();
     if (threadIdx.x == 0) {
         key_s = 0u;
         if (b == 0 && err != nullptr) *err = 0;
     }
     for (int r = threadIdx.x; r < rows_b; r += blockDim.x) {
-        const size_t u0 = ((size_t)b * rows_b + r) * chunks;
+        const size_t gr = (size_t)b * rows_b + r;
+        const size_t u0 = gr * slots;
+        // streamed layout: the row's slots are the warps whose ranges intersect it
+        int chunks = slots;
+        if (vec_per_warp > 0)
+            chunks = (int)(((long long)(gr + 1) * vpr - 1) / vec_per_warp - ((long long)gr * vpr) / vec_per_warp) + 1;
         float best = -INFINITY;
         int arg = 0;   // a row without any value above -inf (all NaN) yields 0
         for (int c = 0; c < chunks; ++c) {
@@ -173,23 +236,44 @@ size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 }  // namespace
 
+// Resident CTAs per SM of the streaming kernel (launch bound above) times the SM count gives the
+// number of warps of one full wave; every warp gets an equal range of at least one unrolled trip.
 VerifyPlan make_verify_plan(int B, int K, int n, int V, int dtype) {
     VerifyPlan p{};
     p.rows = B * K * (n + 1);
     const int esz = dtype == SPEC_BF16 ? 2 : 4;
-    const int gran = 32 * 4 * (16 / esz);   // elements one warp covers per loop trip
-    const long long target_units = (long long)num_sms() * 64 * 2;
-    int chunks = (int)((target_units + p.rows - 1) / p.rows);
-    const int max_chunks = (V + gran - 1) / gran;
-    if (chunks > max_chunks) chunks = max_chunks;
-    if (chunks < 1) chunks = 1;
-    int per = (V + chunks - 1) / chunks;
-    p.chunk_elems = (per + gran - 1) / gran * gran;
-    p.chunks = (V + p.chunk_elems - 1) / p.chunk_elems;
+    const int epv = 16 / esz;
+    // scalar fallback layout (also the upper bound used for the workspace when V % epv != 0)
+    {
+        const int gran = 32 * 4 * epv;
+        const long long target_units = (long long)num_sms() * 64 * 2;
+        int chunks = (int)((target_units + p.rows - 1) / p.rows);
+        const int max_chunks = (V + gran - 1) / gran;
+        if (chunks > max_chunks) chunks = max_chunks;
+        if (chunks < 1) chunks = 1;
+        const int per = (V + chunks - 1) / chunks;
+        p.chunk_elems = (per + gran - 1) / gran * gran;
+        p.chunks = (V + p.chunk_elems - 1) / p.chunk_elems;
+    }
+    p.vpr = 0;
+    p.vec_per_warp = 0;
+    p.slots = p.chunks;
+    if (V % epv == 0) {
+        p.vpr = V / epv;
+        const long long total = (long long)p.rows * p.vpr;
+        const long long wave_warps = (long long)num_sms() * 4 * kWarpsPerBlock;
+        long long c = (total + wave_warps - 1) / wave_warps;
+        const long long min_c = 32 * kStreamUnroll;
+        if (c < min_c) c = min_c;
+        if (c > (1ll << 30)) c = 1ll << 30;
+        p.vec_per_warp = (int)c;
+        const int stream_slots = (int)((p.vpr + c - 1) / c) + 1;
+        if (stream_slots > p.slots) p.slots = stream_slots;
+    }
     p.off_g = kWsAlign;
     p.off_pval = align_up(p.off_g + sizeof(int32_t) * (size_t)p.rows, kWsAlign);
-    p.off_pidx = align_up(p.off_pval + sizeof(float) * (size_t)p.rows * p.chunks, kWsAlign);
-    p.total = align_up(p.off_pidx + sizeof(int32_t) * (size_t)p.rows * p.chunks, kWsAlign);
+    p.off_pidx = align_up(p.off_pval + sizeof(float) * (size_t)p.rows * p.slots, kWsAlign);
+    p.total = align_up(p.off_pidx + sizeof(int32_t) * (size_t)p.rows * p.slots, kWsAlign);
     return p;
 }
 
@@ -201,22 +285,36 @@ int launch_verify(const int32_t *cand_tok, const void *base_logits, int dtype, i
     int32_t *g = (int32_t *)(w + plan.off_g);
     float *pval = (float *)(w + plan.off_pval);
     int32_t *pidx = (int32_t *)(w + plan.off_pidx);
-    const long long units = (long long)plan.rows * plan.chunks;
-    const unsigned grid = (unsigned)((units + kWarpsPerBlock - 1) / kWarpsPerBlock);
-    const int esz = dtype == SPEC_BF16 ? 2 : 4;
-    const bool vec = ((uintptr_t)base_logits % 16 == 0) && (V % (16 / esz) == 0);
-    if (dtype == SPEC_BF16) {
-        if (vec) verify_argmax_kernel<true, true><<<grid, kArgmaxThreads, 0, st>>>(base_logits, plan.rows, V, plan.chunk_elems, plan.chunks, pval, pidx);
-        else verify_argmax_kernel<true, false><<<grid, kArgmaxThreads, 0, st>>>(base_logits, plan.rows, V, plan.chunk_elems, plan.chunks, pval, pidx);
+    const bool stream = plan.vec_per_warp > 0 && ((uintptr_t)base_logits % 16 == 0);
+    int vec_per_warp = 0;
+    if (stream) {
+        vec_per_warp = plan.vec_per_warp;
+        const long long total = (long long)plan.rows * plan.vpr;
+        const long long warps = (total + vec_per_warp - 1) / vec_per_warp;
+        const unsigned grid = (unsigned)((warps + kWarpsPerBlock - 1) / kWarpsPerBlock);
+        const uint4 *lp = (const uint4 *)base_logits;
+        if (dtype == SPEC_BF16)
+            SPEC_CUDA_TRY(launch_pdl(verify_stream_kernel<true>, dim3(grid), dim3(kArgmaxThreads), 0, st, lp, total,
+                                     plan.vpr, vec_per_warp, plan.slots, pval, pidx));
+        else
+            SPEC_CUDA_TRY(launch_pdl(verify_stream_kernel<false>, dim3(grid), dim3(kArgmaxThreads), 0, st, lp, total,
+                                     plan.vpr, vec_per_warp, plan.slots, pval, pidx));
     } else {
-        if (vec) verify_argmax_kernel<false, true><<<grid, kArgmaxThreads, 0, st>>>(base_logits, plan.rows, V, plan.chunk_elems, plan.chunks, pval, pidx);
-        else verify_argmax_kernel<false, false><<<grid, kArgmaxThreads, 0, st>>>(base_logits, plan.rows, V, plan.chunk_elems, plan.chunks, pval, pidx);
+        // scalar fallback; its partials use the first plan.chunks slots of every row, laid out with
+        // plan.chunks as the row pitch
+        const long long units = (long long)plan.rows * plan.chunks;
+        const unsigned grid = (unsigned)((units + kWarpsPerBlock - 1) / kWarpsPerBlock);
+        if (dtype == SPEC_BF16)
+            SPEC_CUDA_TRY(launch_pdl(verify_argmax_kernel<true, false>, dim3(grid), dim3(kArgmaxThreads), 0, st,
+                                     base_logits, plan.rows, V, plan.chunk_elems, plan.chunks, pval, pidx));
+        else
+            SPEC_CUDA_TRY(launch_pdl(verify_argmax_kernel<false, false>, dim3(grid), dim3(kArgmaxThreads), 0, st,
+                                     base_logits, plan.rows, V, plan.chunk_elems, plan.chunks, pval, pidx));
     }
-    SPEC_CUDA_TRY(cudaGetLastError());
     const size_t smem = sizeof(int32_t) * (size_t)K * (n + 1);
-    verify_accept_kernel<<<B, 128, smem, st>>>(cand_tok, pval, pidx, K, n, plan.chunks, g, accept_len, best_cand,
-                                               next_tok, err);
-    SPEC_CUDA_TRY(cudaGetLastError());
+    SPEC_CUDA_TRY(launch_pdl(verify_accept_kernel, dim3(B), dim3(128), smem, st, cand_tok, (const float *)pval,
+                             (const int32_t *)pidx, K, n, stream ? plan.slots : plan.chunks, plan.vpr, vec_per_warp,
+                             g, accept_len, best_cand, next_tok, err));
     return SPEC_OK;
 }
 
