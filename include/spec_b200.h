@@ -38,7 +38,9 @@ enum spec_status {
     SPEC_ERR_TOKEN_RANGE = 5, /* device: a token id was outside [0, V) (its embedding is
                                  treated as zero and the call runs to completion)             */
     SPEC_ERR_TIMEOUT = 6,     /* device: a bounded wait inside a kernel ran out               */
-    SPEC_ERR_NO_DEVICE = 7    /* no CUDA device / not an sm_100 part                          */
+    SPEC_ERR_NO_DEVICE = 7,   /* no CUDA device / not an sm_100 part                          */
+    SPEC_ERR_STATIC_SCRATCH = 8 /* spec_verify_static: the problem needs more scratch than the
+                                 built-in array holds (SPEC_VERIFY_STATIC_SCRATCH_BYTES)      */
 };
 
 enum spec_dtype { SPEC_BF16 = 0, SPEC_F32 = 1 };
@@ -131,6 +133,35 @@ size_t spec_verify_workspace_bytes(int B, int K, int n, int V, int logits_dtype)
 int spec_verify(const int32_t *cand_tok, const void *base_logits, int logits_dtype, int B, int K, int n, int V,
                 int32_t *accept_len, int32_t *best_cand, int32_t *next_tok, void *workspace,
                 size_t workspace_bytes, void *cuda_stream);
+
+/* ---- verify without a caller-supplied workspace -----------------------------------------
+ * (No counterpart in the paper: this is a packaging variant of spec_verify, same results.)
+ * Some hosts of this library cannot hand it scratch memory: a serving process that gave all
+ * of its device memory to its own pools (KV cache, activations) at start-up and must not
+ * grow afterwards, a decode loop that may not take the implicit device-wide stall of an
+ * allocation, or an embedding where another component owns allocation and passes this
+ * library nothing but input and output pointers.  For them the scratch of the verify
+ * kernels (per-row partial maxima and the arg-max table g) lives in an array built into the
+ * library's device image, SPEC_VERIFY_STATIC_SCRATCH_BYTES long; every GPU that loads the
+ * library holds that much memory until the process exits.
+ *   - Arguments and results as spec_verify, minus workspace / workspace_bytes.  No call in
+ *     here allocates or frees memory, on the host or on the device.
+ *   - A problem whose scratch would exceed the array (spec_verify_workspace_bytes(...) >
+ *     SPEC_VERIFY_STATIC_SCRATCH_BYTES) is refused with SPEC_ERR_STATIC_SCRATCH and nothing
+ *     is enqueued.  The five shapes in the benchmark need at most 0.4 MiB.
+ *   - The first call on each device looks up the array's device address (a driver query,
+ *     made with that device current) before it enqueues anything; make that first call
+ *     outside of any stream capture.  Later calls on that device only enqueue kernels.
+ *   - All calls on a device share the one array and it keeps what the last call left there.
+ *     Nothing in it has to be zero beforehand: the kernels overwrite every slot they later
+ *     read and reset the error word themselves.  Two calls whose kernels can overlap on the
+ *     GPU (different streams without an ordering between them) race on the array: order
+ *     them.  The arg-max table g is not reachable by the caller; device-side errors cannot
+ *     occur on this path (it reads no token-indexed memory).
+ */
+#define SPEC_VERIFY_STATIC_SCRATCH_BYTES (1u << 20)
+int spec_verify_static(const int32_t *cand_tok, const void *base_logits, int logits_dtype, int B, int K, int n,
+                       int V, int32_t *accept_len, int32_t *best_cand, int32_t *next_tok, void *cuda_stream);
 
 /* Per-kernel device times of the last spec_draft issued with SPEC_OPT_PROFILE = 1, in launch
  * order: for every head (projection GEMM, mix/LayerNorm/GELU, head GEMM, merge/expand), then

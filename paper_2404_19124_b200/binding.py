@@ -17,7 +17,8 @@ LIB_PATH = os.path.join(_PKG, "libspec_b200.so")
 
 MAX_HEADS, MAX_TOPK, MAX_LEAVES = 8, 8, 4096
 (SPEC_OK, SPEC_ERR_INVALID_ARG, SPEC_ERR_SHAPE, SPEC_ERR_WORKSPACE, SPEC_ERR_CUDA, SPEC_ERR_TOKEN_RANGE,
- SPEC_ERR_TIMEOUT, SPEC_ERR_NO_DEVICE) = range(8)
+ SPEC_ERR_TIMEOUT, SPEC_ERR_NO_DEVICE, SPEC_ERR_STATIC_SCRATCH) = range(9)
+SPEC_VERIFY_STATIC_SCRATCH_BYTES = 1 << 20
 SPEC_BF16, SPEC_F32 = 0, 1
 SPEC_OPT_GEMM_IMPL, SPEC_OPT_HEAD_BLOCK_N, SPEC_OPT_PROJ_BLOCK_N, SPEC_OPT_PROFILE = 0, 1, 2, 3
 
@@ -25,6 +26,7 @@ EXPORTS = [
     "spec_version", "spec_status_str", "spec_last_cuda_error", "spec_create", "spec_destroy", "spec_set_option",
     "spec_draft_workspace_bytes", "spec_draft_layout", "spec_draft", "spec_verify_workspace_bytes", "spec_verify",
     "spec_profile_read", "spec_poll_error", "spec_head_workspace_bytes", "spec_head_logits", "spec_head_topk",
+    "spec_verify_static",
 ]
 
 if not os.path.exists(LIB_PATH):
@@ -71,6 +73,8 @@ _lib.spec_verify_workspace_bytes.restype = C.c_size_t
 _lib.spec_verify_workspace_bytes.argtypes = [C.c_int] * 5
 _lib.spec_verify.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_int, C.c_int, C.c_int,
                              C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]
+_lib.spec_verify_static.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_int, C.c_int, C.c_int,
+                                    C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
 _lib.spec_poll_error.argtypes = [C.c_void_p, C.c_void_p]
 _lib.spec_profile_read.argtypes = [C.c_void_p, C.POINTER(C.c_float), C.c_int, C.POINTER(C.c_int)]
 _lib.spec_head_workspace_bytes.restype = C.c_size_t
@@ -248,6 +252,31 @@ def spec_verify(cand_tok: torch.Tensor, base_logits: torch.Tensor, accept_len: O
     _check(_lib.spec_verify(_ptr(cand_tok), _ptr(base_logits), dt, B, K, n, V, _ptr(outs[0]), _ptr(outs[1]),
                             _ptr(outs[2]), _ptr(workspace), workspace.numel(), _stream_ptr(stream)), "spec_verify")
     return outs[0], outs[1], outs[2], workspace
+
+
+def spec_verify_static(cand_tok: torch.Tensor, base_logits: torch.Tensor, accept_len: torch.Tensor,
+                       best_cand: torch.Tensor, next_tok: torch.Tensor,
+                       stream: Optional[torch.cuda.Stream] = None) -> None:
+    """spec_verify for callers that cannot provide a workspace: the scratch is an array inside the
+    library (SPEC_VERIFY_STATIC_SCRATCH_BYTES).  All three outputs must be passed in (int32 [B], CUDA);
+    this wrapper creates no tensor.  Raises SpecError(SPEC_ERR_STATIC_SCRATCH) when the problem is too
+    large for the array.  Make the first call on a device outside of stream capture; calls that may
+    overlap on the GPU must be ordered by the caller, they share the array."""
+    B, K, n = cand_tok.shape
+    _dev(cand_tok, torch.int32, name="cand_tok")
+    if base_logits.dtype == torch.bfloat16:
+        dt = SPEC_BF16
+    elif base_logits.dtype == torch.float32:
+        dt = SPEC_F32
+    else:
+        raise ValueError("base_logits must be bf16 or fp32")
+    V = base_logits.shape[-1]
+    _dev(base_logits, base_logits.dtype, (B, K, n + 1, V), "base_logits")
+    for t, name in ((accept_len, "accept_len"), (best_cand, "best_cand"), (next_tok, "next_tok")):
+        _dev(t, torch.int32, (B,), name)
+    with torch.cuda.device(cand_tok.device):
+        _check(_lib.spec_verify_static(_ptr(cand_tok), _ptr(base_logits), dt, B, K, n, V, _ptr(accept_len),
+                                       _ptr(best_cand), _ptr(next_tok), _stream_ptr(stream)), "spec_verify_static")
 
 
 def spec_profile_read(h: SpecHandle) -> List[float]:

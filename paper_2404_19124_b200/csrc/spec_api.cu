@@ -183,6 +183,7 @@ const char *spec_status_str(int s) {
         case SPEC_ERR_TOKEN_RANGE: return "token id outside the vocabulary";
         case SPEC_ERR_TIMEOUT: return "bounded wait inside a kernel ran out";
         case SPEC_ERR_NO_DEVICE: return "no usable CUDA device";
+        case SPEC_ERR_STATIC_SCRATCH: return "problem needs more scratch than the library's built-in array holds";
         default: return "unknown status";
     }
 }

@@ -15,6 +15,8 @@
 //   rows into g[b,k,j], counts the matching prefix of every candidate and picks the best one.
 #include <float.h>
 
+#include <mutex>
+
 #include "spec_common.cuh"
 
 namespace spec {
@@ -319,3 +321,49 @@ int launch_verify(const int32_t *cand_tok, const void *base_logits, int dtype, i
 }
 
 }  // namespace spec
+
+// ---- spec_verify_static: the verify scratch lives in the library's own device image ------------
+// For hosts that cannot give the library a workspace (all device memory already committed to their
+// own pools, or no allocation allowed where this runs).  Inside host code the array's name is only a
+// handle for the runtime, not a device address: the address each device mapped it to is asked for
+// once per device with cudaGetSymbolAddress and that pointer is what the kernels receive.
+static __device__ __align__(256) unsigned char g_verify_static_scratch[SPEC_VERIFY_STATIC_SCRATCH_BYTES];
+
+namespace {
+constexpr int kMaxDevices = 64;
+std::mutex g_static_mutex;
+void *g_static_ptr[kMaxDevices] = {};
+}  // namespace
+
+extern "C" int spec_verify_static(const int32_t *cand_tok, const void *base_logits, int logits_dtype, int B, int K,
+                                  int n, int V, int32_t *accept_len, int32_t *best_cand, int32_t *next_tok,
+                                  void *cuda_stream) {
+    using namespace spec;
+    if (!cand_tok || !base_logits || !accept_len || !best_cand || !next_tok) return SPEC_ERR_INVALID_ARG;
+    if (B <= 0 || K <= 0 || n <= 0 || V <= 0) return SPEC_ERR_INVALID_ARG;
+    if (logits_dtype != SPEC_BF16 && logits_dtype != SPEC_F32) return SPEC_ERR_INVALID_ARG;
+    if (K > 65535 || (long long)K * (n + 1) > 12288 || n > 32767) return SPEC_ERR_SHAPE;
+    if ((long long)B * K * (n + 1) > (1ll << 30)) return SPEC_ERR_SHAPE;
+    if (((uintptr_t)base_logits % (logits_dtype == SPEC_BF16 ? 2 : 4)) != 0) return SPEC_ERR_INVALID_ARG;
+    const VerifyPlan plan = make_verify_plan(B, K, n, V, logits_dtype);
+    if (plan.total > (size_t)SPEC_VERIFY_STATIC_SCRATCH_BYTES) return SPEC_ERR_STATIC_SCRATCH;
+
+    int dev = -1;
+    SPEC_CUDA_TRY(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= kMaxDevices) return SPEC_ERR_NO_DEVICE;
+    void *scratch = nullptr;
+    {
+        std::lock_guard<std::mutex> lock(g_static_mutex);
+        if (g_static_ptr[dev] == nullptr) {
+            // first call on this device (which is current): where did this device map the array?
+            void *ptr = nullptr;
+            SPEC_CUDA_TRY(cudaGetSymbolAddress(&ptr, g_verify_static_scratch));
+            if (ptr == nullptr || ((uintptr_t)ptr % kWsAlign) != 0) return SPEC_ERR_WORKSPACE;
+            g_static_ptr[dev] = ptr;
+        }
+        scratch = g_static_ptr[dev];
+    }
+    return launch_verify(cand_tok, base_logits, logits_dtype, B, K, n, V, accept_len, best_cand, next_tok, scratch, plan,
+                         (cudaStream_t)cuda_stream);
+}
+
