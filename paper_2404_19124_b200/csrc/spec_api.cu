@@ -353,7 +353,7 @@ int spec_draft(spec_handle_t h, const void *ctx_state, const int32_t *last_tok, 
         SPEC_PROF_MARK();
         // fold the partials, branch: children (token, cumulative score) of every node
         rc = launch_merge_expand(part_val, part_idx, part_ms, rows, p.lay.n_tiles[l], topk[l], score_l,
-                                 (int32_t *)(ws + p.lay.tok[l + 1]), (float *)(ws + p.lay.score[l + 1]), 0, st);
+                                 (int32_t *)(ws + p.lay.tok[l + 1]), (float *)(ws + p.lay.score[l + 1]), st);
         if (rc != SPEC_OK) return rc;
         SPEC_PROF_MARK();
     }
@@ -452,7 +452,7 @@ int spec_head_topk(spec_handle_t h, int level, const void *states, int rows, int
     int rc = run_head_partials(h, states, h->w.head[level], rows, bn, topk, part_val, part_idx, part_ms,
                                logits_scratch, err, st);
     if (rc != SPEC_OK) return rc;
-    return launch_merge_expand(part_val, part_idx, part_ms, rows, n_tiles, topk, nullptr, tok, logp, 0, st);
+    return launch_merge_expand(part_val, part_idx, part_ms, rows, n_tiles, topk, nullptr, tok, logp, st);
 }
 
 }  // extern "C"

@@ -115,8 +115,7 @@ int launch_mix_ln_gelu(const float *P, int p_splits, size_t p_split_stride, cons
                        const float *gamma, const float *beta, int rows, int d_inner, int V, int parent_div, float a,
                        float b, float eps, void *S_out, int32_t *err, cudaStream_t st);
 int launch_merge_expand(const float *part_val, const int32_t *part_idx, const float *part_ms, int rows, int n_tiles,
-                        int topk, const float *score_in, int32_t *tok_out, float *score_out, int score_is_logp,
-                        cudaStream_t st);
+                        int topk, const float *score_in, int32_t *tok_out, float *score_out, cudaStream_t st);
 struct PruneArgs {
     const int32_t *tok[SPEC_MAX_HEADS]; // tok[l]: tokens of level l+1 nodes
     int32_t topk[SPEC_MAX_HEADS];

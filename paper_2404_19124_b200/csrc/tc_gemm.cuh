@@ -1,0 +1,520 @@
+// Device-side building blocks of the sm_100a tensor-core contraction
+//     C[M, N] = A[M, Kd] * B[N, Kd]^T,  bf16 operands (row-major = K-major for both), fp32 in TMEM,
+// shared by the stand-alone GEMM kernel and by the fused draft kernel.
+//
+// A CTA has 192 threads in three roles that meet only through mbarriers:
+//   warp 0      TMA producer: 128-byte-swizzled [128 x 64] A boxes and [block_n x 64] B boxes into a
+//               ring of shared-memory slots, completion on "full" barriers
+//   warp 1      owns the TMEM allocation; one lane issues tcgen05.mma (M 128, N block_n, K 16) and
+//               commits to the slot's "empty" barrier and, per tile, to "accumulator full"
+//   warps 2-5   epilogue: tcgen05.ld of 32 columns at a time, one thread per accumulator row
+// Two accumulator slots in TMEM let the epilogue of tile i overlap the MMAs of tile i + 1.
+// A "job" is one contraction; its tiles (m fastest, then n, then the K split) are dealt round-robin to
+// the CTAs of the grid, and each role walks the jobs it is given in the same order, carrying its ring
+// position from one job to the next.  Every wait is bounded: when one runs out the CTA records
+// SPEC_ERR_TIMEOUT, raises its abort flag and every role returns false.
+#pragma once
+
+#include <cuda.h>
+
+#include "spec_common.cuh"
+
+namespace spec {
+namespace tc {
+
+constexpr int kBlockM = 128;
+constexpr int kBlockK = 64;            // 64 bf16 = 128 bytes = one swizzle span
+constexpr int kUmmaK = 16;
+constexpr int kThreads = 192;
+constexpr int kEpilogueThreads = 128;  // warps 2-5
+constexpr int kMaxStages = 12;
+constexpr int kABytes = kBlockM * kBlockK * 2;
+constexpr int kSmemLimit = 222 * 1024; // leaves room on the SM for the small kernels that overlap with a GEMM
+constexpr uint32_t kSpinFast = 1u << 14;
+constexpr uint32_t kSpinMax = 1u << 24;
+
+struct __align__(8) Barriers {
+    uint64_t full[kMaxStages];
+    uint64_t empty[kMaxStages];
+    uint64_t acc_full[2];
+    uint64_t acc_empty[2];
+    uint32_t tmem_base;
+    volatile int abort_flag;
+};
+
+// One contraction as the kernels see it.
+struct GemmJob {
+    int M, N, Kd;
+    int block_n, m_tiles, n_tiles;
+    int splits, kb_per_split;   // split-K: tile = (m_tile, n_tile, split), split slowest
+    int w_is_a;                 // 1: A holds the weights (no kernel writes them), B the states; 0: the reverse
+    int first_cta;              // CTA that takes tile 0; tile t goes to CTA (first_cta + t) mod grid
+    GemmEpilogue epi;
+};
+
+// Shared-memory ring and accumulator ring of one CTA.
+struct Pipe {
+    uint8_t *tiles;        // 1024-byte aligned; slot s at tiles + s * slot_bytes: A box, then B box at +kABytes
+    Barriers *bars;
+    uint32_t tmem_base;
+    int stages;
+    uint32_t slot_bytes;
+    int acc_stride;        // TMEM columns between the two accumulator slots
+    int32_t *err;
+};
+
+struct RingPos { int stage; uint32_t phase; };
+struct AccPos { int acc; uint32_t phase; };
+
+__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint64_t *bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
+}
+
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint64_t *bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+
+__device__ __forceinline__ void mbar_arrive(uint64_t *bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+
+__device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(smem_u32(bar)), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+
+// Bounded wait.  Returns false when it gave up (or another role already did).
+__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, Barriers *bars, int32_t *err) {
+    for (uint32_t it = 0; it < kSpinMax; ++it) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if (it > kSpinFast) {
+            if (bars->abort_flag) return false;
+            __nanosleep(64);
+        }
+    }
+    bars->abort_flag = 1;
+    report_error(err, SPEC_ERR_TIMEOUT);
+    return false;
+}
+
+__device__ __forceinline__ void tma_load_2d(void *dst, const CUtensorMap *map, int c0, int c1, uint64_t *bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+        ::"r"(smem_u32(dst)), "l"((uint64_t)map), "r"(c0), "r"(c1), "r"(smem_u32(bar))
+        : "memory");
+}
+
+// Shared-memory matrix descriptor: K-major operand, 128-byte swizzle, rows at a 128-byte
+// pitch, groups of 8 rows 1024 bytes apart (stride byte offset), descriptor version 1.
+__device__ __forceinline__ uint64_t make_smem_desc(uint32_t saddr) {
+    uint64_t d = 0;
+    d |= (uint64_t)((saddr & 0x3ffffu) >> 4);        // start address, bits 0-13
+    d |= (uint64_t)0 << 16;                          // leading byte offset (unused for swizzled K-major)
+    d |= (uint64_t)(1024u >> 4) << 32;               // stride byte offset, bits 32-45
+    d |= (uint64_t)1 << 46;                          // version, bits 46-47
+    d |= (uint64_t)2 << 61;                          // layout type: SWIZZLE_128B
+    return d;
+}
+
+// Instruction descriptor for kind::f16: D = fp32, A = B = bf16, both K-major, M x N tile.
+__device__ __forceinline__ uint32_t make_instr_desc(int m, int n) {
+    uint32_t d = 0;
+    d |= 1u << 4;                      // D format: F32
+    d |= 1u << 7;                      // A format: BF16
+    d |= 1u << 10;                     // B format: BF16
+    d |= (uint32_t)(n >> 3) << 17;     // N / 8
+    d |= (uint32_t)(m >> 4) << 24;     // M / 16
+    return d;
+}
+
+__device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
+                                          uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+
+__device__ __forceinline__ void umma_commit(uint64_t *bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar))
+                 : "memory");
+}
+
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32]) {
+    uint32_t r[32];
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+          "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+          "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr)
+        : "memory");
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+    for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
+}
+
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+__device__ __forceinline__ float ex2_approx(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
+// ---- CTA set-up and tear-down ------------------------------------------------------------------------
+// Called by all threads.  Initialises the barriers, allocates `tmem_cols` TMEM columns (a power of two,
+// at least 32) and returns the pipe description.
+__device__ __forceinline__ Pipe pipe_setup(uint8_t *smem_raw, int stages, uint32_t slot_bytes, int tmem_cols,
+                                           int acc_stride, int32_t *err) {
+    Pipe pp;
+    pp.tiles = (uint8_t *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);   // swizzled tiles: 1024-byte aligned
+    pp.bars = (Barriers *)(pp.tiles + (size_t)stages * slot_bytes);
+    pp.stages = stages;
+    pp.slot_bytes = slot_bytes;
+    pp.acc_stride = acc_stride;
+    pp.err = err;
+    const int warp = threadIdx.x >> 5;
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < stages; ++s) {
+            mbar_init(&pp.bars->full[s], 1);
+            mbar_init(&pp.bars->empty[s], 1);
+        }
+        for (int a = 0; a < 2; ++a) {
+            mbar_init(&pp.bars->acc_full[a], 1);
+            mbar_init(&pp.bars->acc_empty[a], 4);   // one arrival per epilogue warp
+        }
+        pp.bars->abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&pp.bars->tmem_base)),
+                     "r"((uint32_t)tmem_cols)
+                     : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    pp.tmem_base = pp.bars->tmem_base;
+    return pp;
+}
+
+// Called by all threads after every role has left its loops.
+__device__ __forceinline__ void pipe_teardown(const Pipe &pp, int tmem_cols) {
+    __syncwarp();
+    tc_fence_before();
+    __syncthreads();
+    if ((threadIdx.x >> 5) == 1) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(pp.tmem_base), "r"((uint32_t)tmem_cols)
+                     : "memory");
+    }
+}
+
+__device__ __forceinline__ int first_tile_of(const GemmJob &j) {
+    return (int)((blockIdx.x + gridDim.x - (unsigned)j.first_cta % gridDim.x) % gridDim.x);
+}
+
+__device__ __forceinline__ void advance(const Pipe &pp, RingPos &rp) {
+    if (++rp.stage == pp.stages) { rp.stage = 0; rp.phase ^= 1u; }
+}
+
+// ---- producer (one thread) -----------------------------------------------------------------------
+// Loads every k block of this CTA's tiles of job `j`.  The first fill of the ring fetches the weight
+// operand only; then `dep_wait()` is called once (it must return true once the states are readable:
+// the preceding grid has completed, or the grid-wide barrier behind which they are written has
+// opened) and the state operand of those slots follows.  A CTA without a tile in the job neither
+// loads nor waits.  `issued` counts slots filled since the kernel started (for the abort path).
+template <typename DepWait>
+__device__ __forceinline__ bool produce_job(const Pipe &pp, const GemmJob &j, const CUtensorMap *tmap_a,
+                                            const CUtensorMap *tmap_b, RingPos &rp, int &issued, DepWait dep_wait) {
+    const int num_kb = (j.Kd + kBlockK - 1) / kBlockK;
+    const int mn_tiles = j.m_tiles * j.n_tiles;
+    const int num_tiles = mn_tiles * j.splits;
+    const uint32_t tx = (uint32_t)kABytes + (uint32_t)j.block_n * kBlockK * 2;
+    const int first = first_tile_of(j);
+    if (first >= num_tiles) return true;
+    Barriers *bars = pp.bars;
+    int n_pre = 0;
+    {
+        const int split = first / mn_tiles, mn = first - split * mn_tiles;
+        const int m_tile = mn % j.m_tiles, n_tile = mn / j.m_tiles;
+        const int kb0 = split * j.kb_per_split, kb1 = min(num_kb, kb0 + j.kb_per_split);
+        n_pre = min(pp.stages, kb1 - kb0);
+        RingPos q = rp;
+        for (int i = 0; i < n_pre; ++i) {
+            if (!mbar_wait(&bars->empty[q.stage], q.phase ^ 1u, bars, pp.err)) return false;
+            uint8_t *sa = pp.tiles + (size_t)q.stage * pp.slot_bytes;
+            mbar_arrive_expect_tx(&bars->full[q.stage], tx);
+            if (j.w_is_a) tma_load_2d(sa, tmap_a, (kb0 + i) * kBlockK, m_tile * kBlockM, &bars->full[q.stage]);
+            else tma_load_2d(sa + kABytes, tmap_b, (kb0 + i) * kBlockK, n_tile * j.block_n, &bars->full[q.stage]);
+            advance(pp, q);
+        }
+    }
+    if (!dep_wait()) return false;
+    int done = 0;   // k blocks of this job handled so far
+    for (int tile = first; tile < num_tiles; tile += gridDim.x) {
+        const int split = tile / mn_tiles, mn = tile - split * mn_tiles;
+        const int m_tile = mn % j.m_tiles, n_tile = mn / j.m_tiles;
+        const int kb0 = split * j.kb_per_split, kb1 = min(num_kb, kb0 + j.kb_per_split);
+        for (int kb = kb0; kb < kb1; ++kb) {
+            uint8_t *sa = pp.tiles + (size_t)rp.stage * pp.slot_bytes;
+            uint8_t *sb = sa + kABytes;
+            const bool prefetched = done < n_pre;   // the weights of this slot are already on their way
+            if (!prefetched) {
+                if (!mbar_wait(&bars->empty[rp.stage], rp.phase ^ 1u, bars, pp.err)) return false;
+                mbar_arrive_expect_tx(&bars->full[rp.stage], tx);
+            }
+            if (!prefetched || !j.w_is_a) tma_load_2d(sa, tmap_a, kb * kBlockK, m_tile * kBlockM, &bars->full[rp.stage]);
+            if (!prefetched || j.w_is_a) tma_load_2d(sb, tmap_b, kb * kBlockK, n_tile * j.block_n, &bars->full[rp.stage]);
+            ++done;
+            ++issued;
+            advance(pp, rp);
+        }
+    }
+    return true;
+}
+
+// After a failed wait: let the copies already in flight land before the CTA's shared memory is released.
+__device__ __forceinline__ void producer_drain(const Pipe &pp, RingPos rp, int issued) {
+    const int pending = issued < pp.stages ? issued : pp.stages;
+    for (int i = 0; i < pending; ++i) {
+        if (--rp.stage < 0) { rp.stage = pp.stages - 1; rp.phase ^= 1u; }
+        for (uint32_t it = 0; it < (1u << 20) && !mbar_try_wait(&pp.bars->full[rp.stage], rp.phase); ++it) __nanosleep(32);
+    }
+}
+
+// ---- MMA issuer (one thread) ----------------------------------------------------------------------
+__device__ __forceinline__ bool mma_job(const Pipe &pp, const GemmJob &j, RingPos &rp, AccPos &ap) {
+    const int num_kb = (j.Kd + kBlockK - 1) / kBlockK;
+    const int mn_tiles = j.m_tiles * j.n_tiles;
+    const int num_tiles = mn_tiles * j.splits;
+    const uint32_t idesc = make_instr_desc(kBlockM, j.block_n);
+    Barriers *bars = pp.bars;
+    for (int tile = first_tile_of(j); tile < num_tiles; tile += gridDim.x) {
+        if (!mbar_wait(&bars->acc_empty[ap.acc], ap.phase ^ 1u, bars, pp.err)) return false;
+        tc_fence_after();
+        const uint32_t tmem_d = pp.tmem_base + (uint32_t)(ap.acc * pp.acc_stride);
+        const int split = tile / mn_tiles;
+        const int kb0 = split * j.kb_per_split, kb1 = min(num_kb, kb0 + j.kb_per_split);
+        for (int kb = kb0; kb < kb1; ++kb) {
+            if (!mbar_wait(&bars->full[rp.stage], rp.phase, bars, pp.err)) return false;
+            tc_fence_after();
+            const uint32_t sa = smem_u32(pp.tiles + (size_t)rp.stage * pp.slot_bytes);
+            const uint32_t sb = sa + kABytes;
+#pragma unroll
+            for (int k = 0; k < kBlockK / kUmmaK; ++k) {
+                const uint64_t adesc = make_smem_desc(sa + k * kUmmaK * 2);
+                const uint64_t bdesc = make_smem_desc(sb + k * kUmmaK * 2);
+                umma_bf16(tmem_d, adesc, bdesc, idesc, ((kb - kb0) | k) != 0 ? 1u : 0u);
+            }
+            umma_commit(&bars->empty[rp.stage]);   // frees the slot once these MMAs have read it
+            advance(pp, rp);
+        }
+        umma_commit(&bars->acc_full[ap.acc]);
+        if (++ap.acc == 2) { ap.acc = 0; ap.phase ^= 1u; }
+    }
+    return true;
+}
+
+// ---- epilogue, mode 1 -----------------------------------------------------------------------------
+// One thread owns one accumulator row.  Data-dependent insertion into a sorted list diverges in
+// every warp (each lane inserts at different columns), so the selection is done branch-free:
+//   pass 1  streams the tile once: online (max, sum-exp) and the kCap largest VALUES of the row,
+//           kept sorted by a min/max network (new_v[j] = max(v[j], min(v[j-1], x)));
+//   pass 2  re-reads the tile from TMEM and emits the columns whose value reaches the topk-th
+//           largest; equal values are taken in ascending column order, exactly `topk` entries.
+template <int kCap>
+__device__ __forceinline__ void epilogue_topk(const GemmJob &p, uint32_t taddr, int row, bool row_ok, int col0,
+                                              int n_tile) {
+    constexpr float kLog2e = 1.4426950408889634f;
+    float best[kCap];
+#pragma unroll
+    for (int j = 0; j < kCap; ++j) best[j] = -INFINITY;
+    float run_m = -INFINITY, run_s = 0.0f;
+    for (int c = 0; c < p.block_n; c += 32) {
+        float v[32];
+        tmem_ld32(taddr + c, v);
+        const int valid = p.N - (col0 + c);   // columns of this chunk inside the vocabulary
+        if (valid < 32) {
+#pragma unroll
+            for (int i = 0; i < 32; ++i)
+                if (i >= valid) v[i] = -INFINITY;
+        }
+        float cm0 = fmaxf(v[0], v[1]), cm1 = fmaxf(v[2], v[3]);
+#pragma unroll
+        for (int i = 4; i < 32; i += 2) {
+            cm0 = fmaxf(cm0, v[i]);
+            cm1 = fmaxf(cm1, v[i + 1]);
+        }
+        const float cm = fmaxf(cm0, cm1);
+        if (cm > run_m) {
+            run_s *= ex2_approx((run_m - cm) * kLog2e);
+            run_m = cm;
+        }
+        const float ms = run_m * kLog2e;
+        float s0 = 0.0f, s1 = 0.0f, s2 = 0.0f, s3 = 0.0f;
+#pragma unroll
+        for (int i = 0; i < 32; i += 4) {
+            s0 += ex2_approx(fmaf(v[i], kLog2e, -ms));
+            s1 += ex2_approx(fmaf(v[i + 1], kLog2e, -ms));
+            s2 += ex2_approx(fmaf(v[i + 2], kLog2e, -ms));
+            s3 += ex2_approx(fmaf(v[i + 3], kLog2e, -ms));
+        }
+        if (run_m > -INFINITY) run_s += (s0 + s1) + (s2 + s3);
+#pragma unroll
+        for (int i = 0; i < 32; ++i) {
+            const float x = v[i];
+#pragma unroll
+            for (int j = kCap - 1; j > 0; --j) best[j] = fmaxf(best[j], fminf(best[j - 1], x));
+            best[0] = fmaxf(best[0], x);
+        }
+    }
+    // threshold = topk-th largest value of the row in this tile; how many entries lie strictly above it
+    const int topk = p.epi.topk;
+    float thr = best[0];
+#pragma unroll
+    for (int j = 1; j < kCap; ++j)
+        if (j < topk) thr = best[j];
+    int above = 0;
+#pragma unroll
+    for (int j = 0; j < kCap; ++j)
+        if (j < topk && best[j] > thr) ++above;
+    int eq_left = topk - above;
+    const size_t u = (size_t)row * p.n_tiles + n_tile;
+    float *pv = p.epi.part_val + u * SPEC_MAX_TOPK;
+    int32_t *pi = p.epi.part_idx + u * SPEC_MAX_TOPK;
+    int cnt = 0;
+    for (int c = 0; c < p.block_n; c += 32) {
+        float v[32];
+        tmem_ld32(taddr + c, v);
+        const int valid = p.N - (col0 + c);
+        // candidates of this chunk as a bit mask: no per-element branches
+        uint32_t mask = 0;
+#pragma unroll
+        for (int i = 0; i < 32; ++i) mask |= (v[i] >= thr ? 1u : 0u) << i;
+        if (valid < 32) mask &= valid > 0 ? ((1u << valid) - 1u) : 0u;
+        if (!row_ok) mask = 0;
+        while (mask) {   // ascending columns; a handful of iterations per tile
+            const int bpos = __ffs(mask) - 1;
+            mask &= mask - 1;
+            // x = v[bpos] through a select tree (bpos is data dependent, v lives in registers)
+            float t16[16], t8[8], t4[4], t2[2];
+#pragma unroll
+            for (int i = 0; i < 16; ++i) t16[i] = (bpos & 1) ? v[2 * i + 1] : v[2 * i];
+#pragma unroll
+            for (int i = 0; i < 8; ++i) t8[i] = (bpos & 2) ? t16[2 * i + 1] : t16[2 * i];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) t4[i] = (bpos & 4) ? t8[2 * i + 1] : t8[2 * i];
+#pragma unroll
+            for (int i = 0; i < 2; ++i) t2[i] = (bpos & 8) ? t4[2 * i + 1] : t4[2 * i];
+            const float x = (bpos & 16) ? t2[1] : t2[0];
+            const bool gt = x > thr;
+            if (gt || eq_left > 0) {
+                if (!gt) --eq_left;
+                if (cnt < topk) {
+                    pv[cnt] = x;
+                    pi[cnt] = col0 + c + bpos;
+                }
+                ++cnt;
+            }
+        }
+    }
+    if (row_ok) {
+        for (; cnt < topk; ++cnt) {   // fewer than topk comparable values (NaN rows, tiny tiles)
+            pv[cnt] = -INFINITY;
+            pi[cnt] = 0x7fffffff;
+        }
+        p.epi.part_ms[2 * u] = run_m;
+        p.epi.part_ms[2 * u + 1] = run_s;
+    }
+}
+
+// ---- epilogue warps (warps 2-5, all lanes) ----------------------------------------------------------
+__device__ __forceinline__ bool epilogue_job(const Pipe &pp, const GemmJob &j, AccPos &ap) {
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int quarter = warp & 3;               // TMEM lane quarter this warp may read
+    const int row_in_tile = quarter * 32 + lane;
+    const int mn_tiles = j.m_tiles * j.n_tiles;
+    const int num_tiles = mn_tiles * j.splits;
+    Barriers *bars = pp.bars;
+    for (int tile = first_tile_of(j); tile < num_tiles; tile += gridDim.x) {
+        const int split = tile / mn_tiles, mn = tile - split * mn_tiles;
+        const int m_tile = mn % j.m_tiles, n_tile = mn / j.m_tiles;
+        if (!mbar_wait(&bars->acc_full[ap.acc], ap.phase, bars, pp.err)) return false;
+        tc_fence_after();
+        const int row = m_tile * kBlockM + row_in_tile;
+        const bool row_ok = row < j.M;
+        const uint32_t taddr = pp.tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(ap.acc * pp.acc_stride);
+        const int col0 = n_tile * j.block_n;
+        if (j.epi.mode == 0) {
+            for (int c = 0; c < j.block_n; c += 32) {
+                float v[32];
+                tmem_ld32(taddr + c, v);
+                if (row_ok) {
+                    float *dst = j.epi.out + (size_t)row * j.epi.ldc + col0 + c;
+                    const int valid = j.N - (col0 + c);
+                    if (valid >= 32 && (((uintptr_t)dst) & 15) == 0) {
+#pragma unroll
+                        for (int i = 0; i < 32; i += 4)
+                            *(float4 *)(dst + i) = make_float4(v[i], v[i + 1], v[i + 2], v[i + 3]);
+                    } else {
+#pragma unroll
+                        for (int i = 0; i < 32; ++i)
+                            if (i < valid) dst[i] = v[i];
+                    }
+                }
+            }
+        } else if (j.epi.mode == 2) {
+            // transposed store of one split-K partial: out[split][col][row]; a warp's 32 rows are
+            // consecutive addresses, so every store instruction is one 128-byte line
+            float *dst0 = j.epi.out + (size_t)split * j.epi.split_stride + row;
+            for (int c = 0; c < j.block_n; c += 32) {
+                float v[32];
+                tmem_ld32(taddr + c, v);
+                if (row_ok) {
+                    const int valid = j.N - (col0 + c);
+#pragma unroll
+                    for (int i = 0; i < 32; ++i)
+                        if (i < valid) dst0[(size_t)(col0 + c + i) * j.epi.ldc] = v[i];
+                }
+            }
+        } else {
+            if (j.epi.topk <= 4) epilogue_topk<4>(j, taddr, row, row_ok, col0, n_tile);
+            else epilogue_topk<SPEC_MAX_TOPK>(j, taddr, row, row_ok, col0, n_tile);
+        }
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&bars->acc_empty[ap.acc]);
+        if (++ap.acc == 2) { ap.acc = 0; ap.phase ^= 1u; }
+    }
+    return true;
+}
+
+}  // namespace tc
+
+// ---- host side (gemm_tcgen05.cu) ---------------------------------------------------------------
+// 2-D bf16 row-major [rows, cols] tensor, box = [box_rows, 64 columns], 128-byte swizzle; `streamed`
+// marks the operand that is read once from HBM (wider L2 fetches).
+int make_tmap(CUtensorMap *map, const void *base, uint64_t rows, uint64_t cols, uint32_t box_rows, bool streamed);
+// Fills the tiling fields of a job (m_tiles, n_tiles, splits, kb_per_split, w_is_a) from its shape and epilogue.
+int plan_job(tc::GemmJob *j, int M, int N, int Kd, int block_n, const GemmEpilogue &epi);
+
+}  // namespace spec
