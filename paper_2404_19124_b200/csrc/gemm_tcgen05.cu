@@ -54,9 +54,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
             mma_job(pp, p.job, rp, ap);
         }
     } else {
-        griddep_wait();
         AccPos ap{0, 0u};
-        epilogue_job(pp, p.job, ap);
+        epilogue_job(pp, p.job, ap, true);   // real tiles only become ready after the producer's wait
+        griddep_wait();
     }
     pipe_teardown(pp, p.tmem_cols);
 }

@@ -1,14 +1,18 @@
 // Row-wise steps of the draft path (Sec. 3.1 / Sec. 4.1 of arXiv 2404.19124), written for a group of
-// kThreads threads that synchronises through `Sync::sync()`: a whole CTA (__syncthreads) in the
-// stand-alone kernels, the four epilogue warps (a named barrier) inside the fused draft kernel.
+// kThreads threads that synchronises through `Sync::sync()` (a whole CTA in the stand-alone kernels).
 //   mix_ln_gelu_row   embedding gather + weighted mix with the projected parent state (sum of the
 //                     split-K partials) + LayerNorm + exact GELU for one tree node, bf16 state out
 //   merge_expand_row  folds the per-tile partial top-k lists and (max, sum-exp) pairs of one row into
 //                     its top-k tokens and log-probabilities and writes the node's children
 //   prune_sequence    orders one sequence's leaves by (score desc, leaf index asc), keeps K, walks
 //                     back to the root to emit the K n-grams
-// Buffers that an earlier step of the same launch may have written (projections, tokens, scores,
-// partial lists) are read with ld.global.cg, never through the non-coherent path.
+// These steps run once per launch on a handful of rows, so what they cost is latency: round trips
+// to L2 / HBM (all loads of a step are issued before the first is used) and, on an SM that has not
+// run the code yet, instruction fetch (about 0.1 us per 128 bytes of code).  Every step therefore
+// takes a `live` flag: with live == false the same instructions run but nothing produced by an earlier
+// kernel is read and nothing is written, which a kernel uses to pull its code into the instruction
+// cache while it still waits for the kernel before it.
+// Buffers that a preceding kernel wrote are read with ld.global.cg, never through the non-coherent path.
 #pragma once
 
 #include <math.h>
@@ -21,16 +25,12 @@ namespace rows {
 struct BlockSync {
     static __device__ __forceinline__ void sync() { __syncthreads(); }
 };
-template <int kId, int kCount>
-struct NamedSync {
-    static __device__ __forceinline__ void sync() { asm volatile("bar.sync %0, %1;" ::"n"(kId), "n"(kCount) : "memory"); }
-};
 
 // Scratch in shared memory for one group.
 struct Scratch {
     float red[32];
     float red_m[8], red_s[8];
-    float cand_v[2][8];
+    uint32_t cand_k[2][8];
     int cand_i[2][8];
 };
 
@@ -48,7 +48,9 @@ __device__ __forceinline__ float group_sum(float v, float *red, int tid) {
     return t;
 }
 
-__device__ __forceinline__ float gelu_erf(float y) { return 0.5f * y * (1.0f + erff(y * 0.70710678118654752440f)); }
+// Exact (erf) GELU.  erff is kept out of line: inlined it would be the bulk of the row step's code.
+static __device__ __noinline__ float erf_call(float x) { return erff(x); }
+__device__ __forceinline__ float gelu_erf(float y) { return 0.5f * y * (1.0f + erf_call(y * 0.70710678118654752440f)); }
 
 struct MixArgs {
     const float *P;            // `p_splits` partial projections, `p_split_stride` floats apart: [parent rows, d] each
@@ -65,12 +67,15 @@ struct MixArgs {
 
 // Node r of the level.  Siblings share a projected parent state: parent(r) = r / parent_div.
 // h = a * P[parent] + b * E[tok[r]].  The row lives in registers: thread t owns the 8-element groups
-// t, t + kThreads, ... (kIters of them; d <= 8 * kThreads * kIters, d % 8 == 0).
-template <int kThreads, int kIters, typename Sync>
-__device__ __forceinline__ void mix_ln_gelu_row(const MixArgs &m, int r, int tid, float *red) {
-    const int t = __ldcg(m.tok + r);
+// t, t + kThreads, ... (kIters of them; d <= 8 * kThreads * kIters, d % 8 == 0).  kDepth of those
+// groups have their loads in flight together (registers against latency).
+template <int kThreads, int kIters, int kDepth, typename Sync>
+__device__ __forceinline__ void mix_ln_gelu_row(const MixArgs &m, int r, int tid, float *red, bool live) {
+    constexpr int kSp = 4;                                        // partial projections fetched per batch
+    constexpr int kGroup = kIters >= 8 ? 1 : (kIters < kDepth ? kIters : kDepth);
+    const int t = live ? __ldcg(m.tok + r) : 0;
     const bool tok_ok = (t >= 0) && (t < m.V);
-    if (!tok_ok && tid == 0) report_error(m.err, SPEC_ERR_TOKEN_RANGE);
+    if (!tok_ok && tid == 0 && live) report_error(m.err, SPEC_ERR_TOKEN_RANGE);
     const int d = m.d;
     const float *p = m.P + (size_t)(r / m.parent_div) * d;
     const uint16_t *e = m.emb + (size_t)(tok_ok ? t : 0) * d;
@@ -78,27 +83,66 @@ __device__ __forceinline__ void mix_ln_gelu_row(const MixArgs &m, int r, int tid
     float h[kIters][8];
     float sum = 0.0f;
 #pragma unroll
-    for (int it = 0; it < kIters; ++it) {
-        const int i = (it * kThreads + tid) * 8;
+    for (int g0 = 0; g0 < kIters; g0 += kGroup) {
+        // every load of the group is issued before the first value is used: one round trip per group
+        uint4 ev[kGroup];
+        float4 pa[kGroup][kSp], pb[kGroup][kSp];
 #pragma unroll
-        for (int j = 0; j < 8; ++j) h[it][j] = 0.0f;
-        if (i < d) {
-            uint4 ev = make_uint4(0u, 0u, 0u, 0u);
-            if (tok_ok) ev = *(const uint4 *)(e + i);
-            float pv[8] = {0.0f, 0.0f, 0.0f, 0.0f, 0.0f, 0.0f, 0.0f, 0.0f};
-            for (int sp = 0; sp < m.p_splits; ++sp) {
-                const float4 p0 = __ldcg((const float4 *)(p + sp * m.p_split_stride + i));
-                const float4 p1 = __ldcg((const float4 *)(p + sp * m.p_split_stride + i + 4));
-                pv[0] += p0.x; pv[1] += p0.y; pv[2] += p0.z; pv[3] += p0.w;
-                pv[4] += p1.x; pv[5] += p1.y; pv[6] += p1.z; pv[7] += p1.w;
+        for (int q = 0; q < kGroup; ++q) {
+            const int i = ((g0 + q) * kThreads + tid) * 8;
+            ev[q] = make_uint4(0u, 0u, 0u, 0u);
+            if (i < d && tok_ok) ev[q] = *(const uint4 *)(e + i);
+#pragma unroll
+            for (int sp = 0; sp < kSp; ++sp) {
+                pa[q][sp] = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+                pb[q][sp] = pa[q][sp];
+                if (i < d && sp < m.p_splits && live) {
+                    pa[q][sp] = __ldcg((const float4 *)(p + sp * m.p_split_stride + i));
+                    pb[q][sp] = __ldcg((const float4 *)(p + sp * m.p_split_stride + i + 4));
+                }
             }
-            const uint32_t ew[4] = {ev.x, ev.y, ev.z, ev.w};
+        }
+#pragma unroll
+        for (int q = 0; q < kGroup; ++q) {
+            const int it = g0 + q;
+            const int i = (it * kThreads + tid) * 8;
+            float pv[8] = {0.0f, 0.0f, 0.0f, 0.0f, 0.0f, 0.0f, 0.0f, 0.0f};
+#pragma unroll
+            for (int sp = 0; sp < kSp; ++sp) {      // partials are added in ascending order: reproducible
+                pv[0] += pa[q][sp].x; pv[1] += pa[q][sp].y; pv[2] += pa[q][sp].z; pv[3] += pa[q][sp].w;
+                pv[4] += pb[q][sp].x; pv[5] += pb[q][sp].y; pv[6] += pb[q][sp].z; pv[7] += pb[q][sp].w;
+            }
+            if (i < d && live) {
+                for (int sp = kSp; sp < m.p_splits; ++sp) {   // more partials than one batch holds (rare)
+                    const float4 p0 = __ldcg((const float4 *)(p + sp * m.p_split_stride + i));
+                    const float4 p1 = __ldcg((const float4 *)(p + sp * m.p_split_stride + i + 4));
+                    pv[0] += p0.x; pv[1] += p0.y; pv[2] += p0.z; pv[3] += p0.w;
+                    pv[4] += p1.x; pv[5] += p1.y; pv[6] += p1.z; pv[7] += p1.w;
+                }
+            }
+            const uint32_t ew[4] = {ev[q].x, ev[q].y, ev[q].z, ev[q].w};
 #pragma unroll
             for (int j = 0; j < 8; ++j) {
                 const float z = (j & 1) ? __uint_as_float(ew[j >> 1] & 0xffff0000u) : __uint_as_float(ew[j >> 1] << 16);
-                h[it][j] = m.a * pv[j] + m.b * z;
+                h[it][j] = i < d ? m.a * pv[j] + m.b * z : 0.0f;
                 sum += h[it][j];
             }
+        }
+    }
+    // LayerNorm parameters: requested before the two reductions so that they arrive while those run
+    // (for the widest rows they are fetched where they are used, to stay within the register file)
+    constexpr bool kHoist = kIters <= 2;
+    constexpr int kHeld = kHoist ? kIters : 1;
+    float4 gq[kHeld][2], bq[kHeld][2];
+    if (kHoist) {
+#pragma unroll
+        for (int it = 0; it < kHeld; ++it) {
+            const int i = (it * kThreads + tid) * 8;
+            const int ic = i < d ? i : 0;
+            gq[it][0] = *(const float4 *)(m.gamma + ic);
+            gq[it][1] = *(const float4 *)(m.gamma + ic + 4);
+            bq[it][0] = *(const float4 *)(m.beta + ic);
+            bq[it][1] = *(const float4 *)(m.beta + ic + 4);
         }
     }
     const float mean = group_sum<kThreads, Sync>(sum, red, tid) / (float)d;
@@ -119,31 +163,35 @@ __device__ __forceinline__ void mix_ln_gelu_row(const MixArgs &m, int r, int tid
 #pragma unroll
     for (int it = 0; it < kIters; ++it) {
         const int i = (it * kThreads + tid) * 8;
-        if (i < d) {
-            const float4 g0 = *(const float4 *)(m.gamma + i), g1 = *(const float4 *)(m.gamma + i + 4);
-            const float4 b0 = *(const float4 *)(m.beta + i), b1 = *(const float4 *)(m.beta + i + 4);
-            const float gv[8] = {g0.x, g0.y, g0.z, g0.w, g1.x, g1.y, g1.z, g1.w};
-            const float bv[8] = {b0.x, b0.y, b0.z, b0.w, b1.x, b1.y, b1.z, b1.w};
-            uint32_t packed[4];
-#pragma unroll
-            for (int j = 0; j < 8; j += 2) {
-                const float s0 = gelu_erf((h[it][j] - mean) * rstd * gv[j] + bv[j]);
-                const float s1 = gelu_erf((h[it][j + 1] - mean) * rstd * gv[j + 1] + bv[j + 1]);
-                packed[j >> 1] = float_to_bf16_bits(s0) | (float_to_bf16_bits(s1) << 16);
-            }
-            *(uint4 *)(m.S_out + (size_t)r * d + i) = make_uint4(packed[0], packed[1], packed[2], packed[3]);
+        const int hq = kHoist ? it : 0;
+        if (!kHoist) {
+            const int ic = i < d ? i : 0;
+            gq[0][0] = *(const float4 *)(m.gamma + ic);
+            gq[0][1] = *(const float4 *)(m.gamma + ic + 4);
+            bq[0][0] = *(const float4 *)(m.beta + ic);
+            bq[0][1] = *(const float4 *)(m.beta + ic + 4);
         }
+        const float gv[8] = {gq[hq][0].x, gq[hq][0].y, gq[hq][0].z, gq[hq][0].w, gq[hq][1].x, gq[hq][1].y, gq[hq][1].z, gq[hq][1].w};
+        const float bv[8] = {bq[hq][0].x, bq[hq][0].y, bq[hq][0].z, bq[hq][0].w, bq[hq][1].x, bq[hq][1].y, bq[hq][1].z, bq[hq][1].w};
+        uint32_t packed[4];
+#pragma unroll
+        for (int j = 0; j < 8; j += 2) {
+            const float s0 = gelu_erf((h[it][j] - mean) * rstd * gv[j] + bv[j]);
+            const float s1 = gelu_erf((h[it][j + 1] - mean) * rstd * gv[j + 1] + bv[j + 1]);
+            packed[j >> 1] = float_to_bf16_bits(s0) | (float_to_bf16_bits(s1) << 16);
+        }
+        if (i < d && live) *(uint4 *)(m.S_out + (size_t)r * d + i) = make_uint4(packed[0], packed[1], packed[2], packed[3]);
     }
 }
 
 // Picks the register-array size for the row width; false when the row is too wide for this group size.
-template <int kThreads, typename Sync>
-__device__ __forceinline__ bool mix_ln_gelu_row_any(const MixArgs &m, int r, int tid, float *red) {
+template <int kThreads, int kDepth, typename Sync>
+__device__ __forceinline__ bool mix_ln_gelu_row_any(const MixArgs &m, int r, int tid, float *red, bool live) {
     const int groups = (m.d + 8 * kThreads - 1) / (8 * kThreads);
-    if (groups <= 1) mix_ln_gelu_row<kThreads, 1, Sync>(m, r, tid, red);
-    else if (groups <= 2) mix_ln_gelu_row<kThreads, 2, Sync>(m, r, tid, red);
-    else if (groups <= 4) mix_ln_gelu_row<kThreads, 4, Sync>(m, r, tid, red);
-    else if (groups <= 8) mix_ln_gelu_row<kThreads, 8, Sync>(m, r, tid, red);
+    if (groups <= 1) mix_ln_gelu_row<kThreads, 1, kDepth, Sync>(m, r, tid, red, live);
+    else if (groups <= 2) mix_ln_gelu_row<kThreads, 2, kDepth, Sync>(m, r, tid, red, live);
+    else if (groups <= 4) mix_ln_gelu_row<kThreads, 4, kDepth, Sync>(m, r, tid, red, live);
+    else if (groups <= 8) mix_ln_gelu_row<kThreads, 8, kDepth, Sync>(m, r, tid, red, live);
     else return false;
     return true;
 }
@@ -151,8 +199,25 @@ __device__ __forceinline__ bool mix_ln_gelu_row_any(const MixArgs &m, int r, int
 // (value desc, token id asc) ordering of candidates.
 __device__ __forceinline__ bool better(float v, int i, float w, int j) { return v > w || (v == w && i < j); }
 
+// The pair at (va, ia) and the pair at (vb, ib) swap places unless the first is already the better one.
+__device__ __forceinline__ void order_pair(float &va, int &ia, float &vb, int &ib) {
+    if (better(vb, ib, va, ia)) {
+        const float fv = va; va = vb; vb = fv;
+        const int fi = ia; ia = ib; ib = fi;
+    }
+}
+
+// Order-preserving map of a float (no NaN) onto unsigned integers, and back.
+__device__ __forceinline__ uint32_t float_key(float v) {
+    const uint32_t u = __float_as_uint(v);
+    return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
+__device__ __forceinline__ float key_float(uint32_t k) {
+    return __uint_as_float((k & 0x80000000u) ? (k & 0x7fffffffu) : ~k);
+}
+
 struct MergeArgs {
-    const float *part_val;     // [rows, n_tiles, SPEC_MAX_TOPK] (first `topk` of each list valid, best first)
+    const float *part_val;     // [rows, n_tiles, SPEC_MAX_TOPK] (first `topk` of each list valid, any order)
     const int32_t *part_idx;   // same shape
     const float *part_ms;      // [rows, n_tiles, 2] = (max, sum of exp(x - max))
     int n_tiles, topk;
@@ -161,52 +226,97 @@ struct MergeArgs {
     float *score_out;          // [rows, topk]
 };
 
-// Thread t folds the lists of tiles t, t + kThreads, ... into a sorted list in registers with all of
-// its loads independent of one another; the group then extracts the `topk` best in `topk` rounds of
-// (warp arg-max by shuffles, one shared-memory exchange between the warps).
-template <int kThreads, typename Sync>
-__device__ __forceinline__ void merge_expand_row(const MergeArgs &g, int r, int tid, Scratch *sc) {
-    constexpr int kWarps = kThreads / 32;
-    const int lane = tid & 31, warp = tid >> 5;
-    const int n_tiles = g.n_tiles, topk = g.topk;
-    const float4 *pv4 = (const float4 *)(g.part_val + (size_t)r * n_tiles * SPEC_MAX_TOPK);
-    const int4 *pi4 = (const int4 *)(g.part_idx + (size_t)r * n_tiles * SPEC_MAX_TOPK);
-    const float2 *pms = (const float2 *)(g.part_ms + (size_t)r * n_tiles * 2);
-
-    float tv[SPEC_MAX_TOPK];
-    int ti[SPEC_MAX_TOPK];
+// Sorts one tile's list (8 slots, any order, slots >= topk ignored) best first with a fixed network and
+// folds it into the sorted list (tv, ti): with both lists sorted, "the better of a[i] and b[7 - i]" keeps
+// the best 8 of the 16 as a bitonic sequence, which three compare-exchange stages sort (depth 10 in all,
+// where an insertion chain has 64).
+__device__ __forceinline__ void fold_tile_list(float (&tv)[SPEC_MAX_TOPK], int (&ti)[SPEC_MAX_TOPK], const float4 &v0,
+                                               const float4 &v1, const int4 &i0, const int4 &i1, int topk, bool valid) {
+    constexpr int kT = SPEC_MAX_TOPK;
+    static_assert(kT == 8, "the networks are written for lists of 8");
+    float lv[kT] = {v0.x, v0.y, v0.z, v0.w, v1.x, v1.y, v1.z, v1.w};
+    int li[kT] = {i0.x, i0.y, i0.z, i0.w, i1.x, i1.y, i1.z, i1.w};
 #pragma unroll
-    for (int j = 0; j < SPEC_MAX_TOPK; ++j) {
+    for (int j = 0; j < kT; ++j) {
+        if (j >= topk || !valid) {   // slots past the list's length hold nothing
+            lv[j] = -INFINITY;
+            li[j] = 0x7fffffff;
+        }
+    }
+    // 19-comparator sorting network for 8 inputs
+#define SPEC_CX(a, b) order_pair(lv[a], li[a], lv[b], li[b])
+    SPEC_CX(0, 2); SPEC_CX(1, 3); SPEC_CX(4, 6); SPEC_CX(5, 7);
+    SPEC_CX(0, 4); SPEC_CX(1, 5); SPEC_CX(2, 6); SPEC_CX(3, 7);
+    SPEC_CX(0, 1); SPEC_CX(2, 3); SPEC_CX(4, 5); SPEC_CX(6, 7);
+    SPEC_CX(2, 4); SPEC_CX(3, 5);
+    SPEC_CX(1, 4); SPEC_CX(3, 6);
+    SPEC_CX(1, 2); SPEC_CX(3, 4); SPEC_CX(5, 6);
+#undef SPEC_CX
+#pragma unroll
+    for (int j = 0; j < kT; ++j) {
+        if (better(lv[kT - 1 - j], li[kT - 1 - j], tv[j], ti[j])) {
+            tv[j] = lv[kT - 1 - j];
+            ti[j] = li[kT - 1 - j];
+        }
+    }
+#pragma unroll
+    for (int stride = kT / 2; stride > 0; stride >>= 1) {
+#pragma unroll
+        for (int j = 0; j < kT; ++j)
+            if ((j & stride) == 0) order_pair(tv[j], ti[j], tv[j + stride], ti[j + stride]);
+    }
+}
+
+__device__ __forceinline__ void fold_max_sum(float &m, float &s, const float2 &ms) {
+    if (ms.x > m) {
+        s = s * __expf(m - ms.x) + ms.y;   // exp(-inf) = 0 on the first tile
+        m = ms.x;
+    } else if (ms.x > -INFINITY) {
+        s += ms.y * __expf(ms.x - m);
+    }
+}
+
+// Thread t folds the lists of tiles t, t + kThreads, ... into one sorted list of 8 in registers, two
+// tiles per trip with all ten loads issued before the first is used.  The group then extracts the `topk`
+// best in `topk` rounds; a round is two warp-wide integer reductions (redux.sync: maximum of the value
+// keys, then minimum token id among the lanes that hold it) and one shared-memory exchange between warps.
+template <int kThreads, typename Sync>
+__device__ __forceinline__ void merge_expand_row(const MergeArgs &g, int r, int tid, Scratch *sc, bool live) {
+    constexpr int kWarps = kThreads / 32;
+    constexpr int kT = SPEC_MAX_TOPK;
+    const int lane = tid & 31, warp = tid >> 5;
+    const int n_tiles = live ? g.n_tiles : min(g.n_tiles, 1), topk = g.topk;
+    const float4 *pv4 = (const float4 *)(g.part_val + (size_t)r * g.n_tiles * kT);
+    const int4 *pi4 = (const int4 *)(g.part_idx + (size_t)r * g.n_tiles * kT);
+    const float2 *pms = (const float2 *)(g.part_ms + (size_t)r * g.n_tiles * 2);
+    const float base = (g.score_in && live) ? __ldcg(g.score_in + r) : 0.0f;
+
+    float tv[kT];
+    int ti[kT];
+#pragma unroll
+    for (int j = 0; j < kT; ++j) {
         tv[j] = -INFINITY;
         ti[j] = 0x7fffffff;
     }
     float m = -INFINITY, s = 0.0f;
-    for (int t = tid; t < n_tiles; t += kThreads) {
-        const float2 ms = __ldcg(pms + t);
-        const float4 v0 = __ldcg(pv4 + 2 * t), v1 = __ldcg(pv4 + 2 * t + 1);
-        const int4 i0 = __ldcg(pi4 + 2 * t), i1 = __ldcg(pi4 + 2 * t + 1);
-        if (ms.x > m) {
-            s = s * __expf(m - ms.x) + ms.y;   // exp(-inf) = 0 on the first tile
-            m = ms.x;
-        } else if (ms.x > -INFINITY) {
-            s += ms.y * __expf(ms.x - m);
+    for (int t = tid; t < n_tiles; t += 2 * kThreads) {
+        const int t2 = t + kThreads;
+        const bool has2 = t2 < n_tiles;
+        const int tb = has2 ? t2 : t;
+        float2 ms_a = make_float2(-INFINITY, 0.0f), ms_b = ms_a;
+        float4 va0 = make_float4(0.f, 0.f, 0.f, 0.f), va1 = va0, vb0 = va0, vb1 = va0;
+        int4 ia0 = make_int4(0, 1, 2, 3), ia1 = make_int4(4, 5, 6, 7), ib0 = ia0, ib1 = ia1;
+        if (live) {
+            ms_a = __ldcg(pms + t); ms_b = __ldcg(pms + tb);
+            va0 = __ldcg(pv4 + 2 * t); va1 = __ldcg(pv4 + 2 * t + 1);
+            ia0 = __ldcg(pi4 + 2 * t); ia1 = __ldcg(pi4 + 2 * t + 1);
+            vb0 = __ldcg(pv4 + 2 * tb); vb1 = __ldcg(pv4 + 2 * tb + 1);
+            ib0 = __ldcg(pi4 + 2 * tb); ib1 = __ldcg(pi4 + 2 * tb + 1);
         }
-        const float lv[8] = {v0.x, v0.y, v0.z, v0.w, v1.x, v1.y, v1.z, v1.w};
-        const int li[8] = {i0.x, i0.y, i0.z, i0.w, i1.x, i1.y, i1.z, i1.w};
-#pragma unroll
-        for (int j = 0; j < SPEC_MAX_TOPK; ++j) {
-            if (j < topk && better(lv[j], li[j], tv[SPEC_MAX_TOPK - 1], ti[SPEC_MAX_TOPK - 1])) {
-                tv[SPEC_MAX_TOPK - 1] = lv[j];
-                ti[SPEC_MAX_TOPK - 1] = li[j];
-#pragma unroll
-                for (int q = SPEC_MAX_TOPK - 1; q > 0; --q) {
-                    if (better(tv[q], ti[q], tv[q - 1], ti[q - 1])) {
-                        const float fv = tv[q]; tv[q] = tv[q - 1]; tv[q - 1] = fv;
-                        const int fi = ti[q]; ti[q] = ti[q - 1]; ti[q - 1] = fi;
-                    }
-                }
-            }
-        }
+        fold_max_sum(m, s, ms_a);
+        if (has2) fold_max_sum(m, s, ms_b);
+        fold_tile_list(tv, ti, va0, va1, ia0, ia1, topk, true);
+        fold_tile_list(tv, ti, vb0, vb1, ib0, ib1, topk, has2);
     }
     // log-sum-exp of the whole row
     float wm = m;
@@ -215,7 +325,7 @@ __device__ __forceinline__ void merge_expand_row(const MergeArgs &g, int r, int 
     float ws = (m > -INFINITY) ? s * __expf(m - wm) : 0.0f;
 #pragma unroll
     for (int off = 16; off > 0; off >>= 1) ws += __shfl_xor_sync(0xffffffffu, ws, off);
-    Sync::sync();   // the scratch may still be read by the previous row's last round
+    Sync::sync();   // the scratch may still be read by a previous call's last round
     if (lane == 0) {
         sc->red_m[warp] = wm;
         sc->red_s[warp] = ws;
@@ -230,47 +340,38 @@ __device__ __forceinline__ void merge_expand_row(const MergeArgs &g, int r, int 
         if (sc->red_m[w] > -INFINITY) bs += sc->red_s[w] * __expf(sc->red_m[w] - bm);
     const float lse = bm + logf(bs);
 
-    const float base = g.score_in ? __ldcg(g.score_in + r) : 0.0f;
     for (int j = 0; j < topk; ++j) {
-        float bv = tv[0];
-        int bi = ti[0];
-#pragma unroll
-        for (int off = 16; off > 0; off >>= 1) {
-            const float ov = __shfl_xor_sync(0xffffffffu, bv, off);
-            const int oi = __shfl_xor_sync(0xffffffffu, bi, off);
-            if (better(ov, oi, bv, bi)) {
-                bv = ov;
-                bi = oi;
-            }
-        }
+        const uint32_t my_key = float_key(tv[0]);
+        const uint32_t wk = __reduce_max_sync(0xffffffffu, my_key);
+        const uint32_t wi = __reduce_min_sync(0xffffffffu, my_key == wk ? (uint32_t)ti[0] : 0xffffffffu);
         if (lane == 0) {
-            sc->cand_v[j & 1][warp] = bv;
-            sc->cand_i[j & 1][warp] = bi;
+            sc->cand_k[j & 1][warp] = wk;
+            sc->cand_i[j & 1][warp] = (int)wi;
         }
         Sync::sync();   // rounds alternate between two buffers, so one barrier per round is enough
-        bv = sc->cand_v[j & 1][0];
-        bi = sc->cand_i[j & 1][0];
+        uint32_t bk = sc->cand_k[j & 1][0];
+        int bi = sc->cand_i[j & 1][0];
 #pragma unroll
         for (int w = 1; w < kWarps; ++w) {
-            const float ov = sc->cand_v[j & 1][w];
+            const uint32_t ok = sc->cand_k[j & 1][w];
             const int oi = sc->cand_i[j & 1][w];
-            if (better(ov, oi, bv, bi)) {
-                bv = ov;
+            if (ok > bk || (ok == bk && oi < bi)) {
+                bk = ok;
                 bi = oi;
             }
         }
-        if (ti[0] == bi && tv[0] == bv) {   // token ids are unique, so exactly one thread owns a real entry
+        if (ti[0] == bi && my_key == bk) {   // token ids are unique, so exactly one thread owns a real entry
 #pragma unroll
-            for (int q = 0; q < SPEC_MAX_TOPK - 1; ++q) {
+            for (int q = 0; q < kT - 1; ++q) {
                 tv[q] = tv[q + 1];
                 ti[q] = ti[q + 1];
             }
-            tv[SPEC_MAX_TOPK - 1] = -INFINITY;
-            ti[SPEC_MAX_TOPK - 1] = 0x7fffffff;
+            tv[kT - 1] = -INFINITY;
+            ti[kT - 1] = 0x7fffffff;
         }
-        if (tid == 0) {
+        if (tid == 0 && live) {
             g.tok_out[(size_t)r * topk + j] = bi;
-            g.score_out[(size_t)r * topk + j] = base + (bv - lse);
+            g.score_out[(size_t)r * topk + j] = base + (key_float(bk) - lse);
         }
     }
 }
@@ -284,17 +385,42 @@ __device__ __forceinline__ bool leaf_before(const LeafKey &a, const LeafKey &b) 
     return a.score > b.score || (a.score == b.score && a.leaf < b.leaf);
 }
 
-// Sequence b: bitonic sort of the (score, leaf) keys in shared memory (`keys`: Lpad entries, Lpad the
-// power of two >= max(L, 2)), then the K best leaves are traced back to the root.
+// Writes candidate `rank` of sequence b: its score and the tokens on the path from the root to `leaf`.
+__device__ __forceinline__ void emit_candidate(const PruneArgs &pa, int L, int K, int32_t *cand_tok, float *cand_logp,
+                                               int b, int rank, float score, int leaf, bool live) {
+    if (live) cand_logp[(size_t)b * K + rank] = score;
+    int idx = leaf;            // index among this sequence's nodes of level n
+    int per_seq = L;           // nodes of this sequence at level l + 1
+    for (int l = pa.n - 1; l >= 0; --l) {
+        if (live) cand_tok[((size_t)b * K + rank) * pa.n + l] = __ldcg(pa.tok[l] + (size_t)b * per_seq + idx);
+        idx /= pa.topk[l];
+        per_seq /= pa.topk[l];
+    }
+}
+
+// Sequence b: the K best leaves by (score desc, leaf index asc), traced back to the root.  `keys`:
+// shared memory for Lpad entries, Lpad the power of two >= max(L, 2).  Up to 256 leaves every thread
+// counts how many leaves precede its own (that is its rank; no barriers); longer lists are sorted
+// bitonically.
 template <int kThreads, typename Sync>
 __device__ __forceinline__ void prune_sequence(const float *leaf_score, const PruneArgs &pa, int L, int Lpad, int K,
-                                               int32_t *cand_tok, float *cand_logp, int b, int tid, LeafKey *keys) {
-    Sync::sync();   // the previous sequence's back-trace still reads the keys
+                                               int32_t *cand_tok, float *cand_logp, int b, int tid, LeafKey *keys,
+                                               bool live) {
+    Sync::sync();   // a previous call may still be reading the keys
     for (int i = tid; i < Lpad; i += kThreads) {
-        keys[i].score = i < L ? __ldcg(leaf_score + (size_t)b * L + i) : -INFINITY;
+        keys[i].score = (i < L && live) ? __ldcg(leaf_score + (size_t)b * L + i) : -INFINITY;
         keys[i].leaf = i < L ? i : 0x7fffffff;
     }
     Sync::sync();
+    if (L <= 256) {
+        for (int i = tid; i < L; i += kThreads) {
+            const LeafKey mine = keys[i];
+            int rank = 0;
+            for (int j = 0; j < L; ++j) rank += leaf_before(keys[j], mine) ? 1 : 0;
+            if (rank < K) emit_candidate(pa, L, K, cand_tok, cand_logp, b, rank, mine.score, mine.leaf, live);
+        }
+        return;
+    }
     for (int size = 2; size <= Lpad; size <<= 1) {
         for (int stride = size >> 1; stride > 0; stride >>= 1) {
             for (int i = tid; i < Lpad / 2; i += kThreads) {
@@ -311,17 +437,8 @@ __device__ __forceinline__ void prune_sequence(const float *leaf_score, const Pr
             Sync::sync();
         }
     }
-    for (int k = tid; k < K; k += kThreads) {
-        const LeafKey kk = keys[k];
-        cand_logp[(size_t)b * K + k] = kk.score;
-        int idx = kk.leaf;         // index among this sequence's nodes of level n
-        int per_seq = L;           // nodes of this sequence at level l + 1
-        for (int l = pa.n - 1; l >= 0; --l) {
-            cand_tok[((size_t)b * K + k) * pa.n + l] = __ldcg(pa.tok[l] + (size_t)b * per_seq + idx);
-            idx /= pa.topk[l];
-            per_seq /= pa.topk[l];
-        }
-    }
+    for (int k = tid; k < K; k += kThreads)
+        emit_candidate(pa, L, K, cand_tok, cand_logp, b, k, keys[k].score, keys[k].leaf, live);
 }
 
 }  // namespace rows
