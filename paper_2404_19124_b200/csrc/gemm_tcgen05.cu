@@ -22,18 +22,24 @@ namespace {
 
 using namespace tc;
 
+constexpr int kMaxJobs = 2;
+
 struct GemmParams {
-    GemmJob job;
-    int stages, tmem_cols;
+    GemmJob job[kMaxJobs];   // walked in order by every role; both read only what the preceding grid produced
+    int n_jobs;
+    int stages, tmem_cols, acc_stride;
     uint32_t slot_bytes;
     int32_t *err;
 };
 
+struct GemmMaps {
+    CUtensorMap a[kMaxJobs], b[kMaxJobs];
+};
+
 __global__ void __launch_bounds__(kThreads, 1)
-gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
-               const GemmParams p) {
+gemm_tc_kernel(const __grid_constant__ GemmMaps maps, const __grid_constant__ GemmParams p) {
     extern __shared__ uint8_t smem_raw[];
-    const Pipe pp = pipe_setup(smem_raw, p.stages, p.slot_bytes, p.tmem_cols, p.job.block_n, p.err);
+    const Pipe pp = pipe_setup(smem_raw, p.stages, p.slot_bytes, p.tmem_cols, p.acc_stride, p.err);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
     griddep_launch();   // the next kernel in the stream may start its own set-up now
@@ -41,9 +47,11 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
         if (lane == 0) {
             RingPos rp{0, 0u};
             int issued = 0;
+            bool ok = true;
             // the weights are fetched before the preceding grid is waited for, the states after
-            if (!produce_job(pp, p.job, &tmap_a, &tmap_b, rp, issued, [] { griddep_wait(); return true; }))
-                producer_drain(pp, rp, issued);
+            for (int q = 0; ok && q < p.n_jobs; ++q)
+                ok = produce_job(pp, p.job[q], &maps.a[q], &maps.b[q], rp, issued, [] { griddep_wait(); return true; });
+            if (!ok) producer_drain(pp, rp, issued);
         }
         griddep_wait();
     } else if (warp == 1) {
@@ -51,11 +59,14 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
         if (lane == 0) {
             RingPos rp{0, 0u};
             AccPos ap{0, 0u};
-            mma_job(pp, p.job, rp, ap);
+            bool ok = true;
+            for (int q = 0; ok && q < p.n_jobs; ++q) ok = mma_job(pp, p.job[q], rp, ap);
         }
     } else {
         AccPos ap{0, 0u};
-        epilogue_job(pp, p.job, ap, true);   // real tiles only become ready after the producer's wait
+        bool ok = true;
+        // real tiles only become ready after the producer's wait; the dry pass of the first job comes before it
+        for (int q = 0; ok && q < p.n_jobs; ++q) ok = epilogue_job(pp, p.job[q], ap, q == 0);
         griddep_wait();
     }
     pipe_teardown(pp, p.tmem_cols);
@@ -139,26 +150,42 @@ int plan_job(tc::GemmJob *j, int M, int N, int Kd, int block_n, const GemmEpilog
     return SPEC_OK;
 }
 
-int launch_gemm_tc(const void *A, const void *B, int M, int N, int Kd, int block_n, const GemmEpilogue &epi,
-                   int32_t *err, cudaStream_t st) {
+// One launch, one or two contractions.  The tiles of the second are dealt to the CTAs starting where
+// the first one's stopped, so a CTA that got no tile of the first starts on the second at once.
+int launch_gemm_tc_jobs(const GemmCall *calls, int n_calls, int32_t *err, cudaStream_t st) {
+    if (n_calls < 1 || n_calls > kMaxJobs) return SPEC_ERR_INVALID_ARG;
     GemmParams p{};
-    int rc = plan_job(&p.job, M, N, Kd, block_n, epi);
-    if (rc != SPEC_OK) return rc;
-    if (((uintptr_t)A & 15) || ((uintptr_t)B & 15)) return SPEC_ERR_INVALID_ARG;
-    CUtensorMap ta, tb;
-    rc = make_tmap(&ta, A, (uint64_t)M, (uint64_t)Kd, kBlockM, p.job.w_is_a != 0);
-    if (rc != SPEC_OK) return rc;
-    rc = make_tmap(&tb, B, (uint64_t)N, (uint64_t)Kd, (uint32_t)block_n, p.job.w_is_a == 0);
-    if (rc != SPEC_OK) return rc;
-
-    p.slot_bytes = (uint32_t)kABytes + (uint32_t)block_n * kBlockK * 2;
+    GemmMaps maps{};
+    p.n_jobs = n_calls;
+    int max_block_n = 32;
+    long long total_tiles = 0;
+    for (int q = 0; q < n_calls; ++q) {
+        const GemmCall &c = calls[q];
+        int rc = plan_job(&p.job[q], c.M, c.N, c.Kd, c.block_n, c.epi);
+        if (rc != SPEC_OK) return rc;
+        if (((uintptr_t)c.A & 15) || ((uintptr_t)c.B & 15)) return SPEC_ERR_INVALID_ARG;
+        rc = make_tmap(&maps.a[q], c.A, (uint64_t)c.M, (uint64_t)c.Kd, kBlockM, p.job[q].w_is_a != 0);
+        if (rc != SPEC_OK) return rc;
+        rc = make_tmap(&maps.b[q], c.B, (uint64_t)c.N, (uint64_t)c.Kd, (uint32_t)c.block_n, p.job[q].w_is_a == 0);
+        if (rc != SPEC_OK) return rc;
+        if (c.block_n > max_block_n) max_block_n = c.block_n;
+        total_tiles += (long long)p.job[q].m_tiles * p.job[q].n_tiles * p.job[q].splits;
+    }
+    const int grid = (int)(total_tiles < num_sms() ? total_tiles : num_sms());
+    long long offset = 0;
+    for (int q = 0; q < n_calls; ++q) {
+        p.job[q].first_cta = (int)(offset % grid);
+        offset += (long long)p.job[q].m_tiles * p.job[q].n_tiles * p.job[q].splits;
+    }
+    p.slot_bytes = (uint32_t)kABytes + (uint32_t)max_block_n * kBlockK * 2;
     const int budget = kSmemLimit - 1024 - (int)sizeof(Barriers) - 64;
     p.stages = budget / (int)p.slot_bytes;
     if (p.stages > kMaxStages) p.stages = kMaxStages;
     if (p.stages < 2) return SPEC_ERR_SHAPE;
     int cols = 32;
-    while (cols < 2 * block_n) cols <<= 1;
+    while (cols < 2 * max_block_n) cols <<= 1;
     p.tmem_cols = cols;
+    p.acc_stride = max_block_n;
     p.err = err;
 
     const size_t smem = 1024 + (size_t)p.stages * p.slot_bytes + sizeof(Barriers);
@@ -169,10 +196,14 @@ int launch_gemm_tc(const void *A, const void *B, int M, int N, int Kd, int block
         SPEC_CUDA_TRY(cudaFuncSetAttribute(gemm_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemLimit));
         if (dev >= 0 && dev < 64) attr_set[dev] = true;
     }
-    const long long tiles = (long long)p.job.m_tiles * p.job.n_tiles * p.job.splits;
-    const int grid = (int)(tiles < num_sms() ? tiles : num_sms());
-    SPEC_CUDA_TRY(launch_pdl(gemm_tc_kernel, dim3(grid), dim3(kThreads), smem, st, ta, tb, p));
+    SPEC_CUDA_TRY(launch_pdl(gemm_tc_kernel, dim3(grid), dim3(kThreads), smem, st, maps, p));
     return SPEC_OK;
+}
+
+int launch_gemm_tc(const void *A, const void *B, int M, int N, int Kd, int block_n, const GemmEpilogue &epi,
+                   int32_t *err, cudaStream_t st) {
+    GemmCall c{A, B, M, N, Kd, block_n, epi};
+    return launch_gemm_tc_jobs(&c, 1, err, st);
 }
 
 }  // namespace spec

@@ -315,6 +315,31 @@ int spec_draft(spec_handle_t h, const void *ctx_state, const int32_t *last_tok, 
     float *part_ms = (float *)(ws + p.lay.part_ms);
     float *logits_scratch = (float *)(ws + p.lay.logits);
 
+    // state projection of level l as a tensor-core contraction: with few parent rows the weights take
+    // the 128-row side and split-K partials are stored transposed, otherwise the plain form
+    auto proj_call = [&](int l) {
+        const int parent_rows = l == 0 ? B : p.N[l - 1];
+        const void *parent_states = l == 0 ? ctx_state : (const void *)(ws + p.lay.state[l - 1]);
+        GemmCall c{};
+        c.Kd = d_in_of(w, l);
+        c.epi.out = P;
+        c.epi.ldc = w.d_inner;
+        if (p.proj_splits[l] > 0) {
+            c.A = w.proj[l]; c.M = w.d_inner;
+            c.B = parent_states; c.N = parent_rows;
+            c.block_n = (parent_rows + 31) / 32 * 32;
+            c.epi.mode = 2;
+            c.epi.splits = p.proj_splits[l];
+            c.epi.split_stride = (size_t)parent_rows * w.d_inner;
+        } else {
+            c.A = parent_states; c.M = parent_rows;
+            c.B = w.proj[l]; c.N = w.d_inner;
+            c.block_n = p.proj_block_n[l];
+            c.epi.mode = 0;
+        }
+        return c;
+    };
+    bool proj_done = false;   // the projection of the level about to start ran with the previous head
     for (int l = 0; l < p.n; ++l) {
         const int rows = p.N[l];
         const int parent_rows = l == 0 ? B : p.N[l - 1];
@@ -322,23 +347,20 @@ int spec_draft(spec_handle_t h, const void *ctx_state, const int32_t *last_tok, 
         const int32_t *tok_l = l == 0 ? last_tok : (const int32_t *)(ws + p.lay.tok[l]);
         const float *score_l = l == 0 ? nullptr : (const float *)(ws + p.lay.score[l]);
         void *S = ws + p.lay.state[l];
-        // projection of every distinct parent state: P = S_parent * Wp^T
+        // projection of every distinct parent state: P = S_parent * Wp^T (unless it already ran in the
+        // same launch as the previous level's head, see below)
         const int splits = p.proj_splits[l];
         const size_t split_stride = (size_t)parent_rows * w.d_inner;
-        if (splits > 0) {
-            GemmEpilogue e{};
-            e.mode = 2;
-            e.out = P;
-            e.ldc = w.d_inner;
-            e.splits = splits;
-            e.split_stride = split_stride;
-            rc = launch_gemm_tc(w.proj[l], parent_states, w.d_inner, parent_rows, d_in_of(w, l),
-                                (parent_rows + 31) / 32 * 32, e, err, st);
-        } else {
-            rc = run_gemm_store(h, parent_states, w.proj[l], parent_rows, w.d_inner, d_in_of(w, l),
-                                p.proj_block_n[l], P, err, st);
+        if (!proj_done) {
+            if (h->gemm_impl == 0) {
+                const GemmCall c = proj_call(l);
+                rc = launch_gemm_tc_jobs(&c, 1, err, st);
+            } else {
+                rc = run_gemm_store(h, parent_states, w.proj[l], parent_rows, w.d_inner, d_in_of(w, l),
+                                    p.proj_block_n[l], P, err, st);
+            }
+            if (rc != SPEC_OK) return rc;
         }
-        if (rc != SPEC_OK) return rc;
         SPEC_PROF_MARK();
         // gather + mix + LayerNorm + GELU -> bf16 state of every node of this level
         rc = launch_mix_ln_gelu(P, splits > 0 ? splits : 1, split_stride, w.emb[l], tok_l, w.ln_gamma[l],
@@ -346,9 +368,26 @@ int spec_draft(spec_handle_t h, const void *ctx_state, const int32_t *last_tok, 
                                 w.emb_weight, w.ln_eps, S, err, st);
         if (rc != SPEC_OK) return rc;
         SPEC_PROF_MARK();
-        // vocabulary head with the fused per-tile top-k / log-sum-exp epilogue
-        rc = run_head_partials(h, S, w.head[l], rows, p.lay.block_n[l], topk[l], part_val, part_idx, part_ms,
-                               logits_scratch, err, st);
+        // vocabulary head with the fused per-tile top-k / log-sum-exp epilogue.  The next level's
+        // projection needs nothing newer than this level's states either, so it rides in the same
+        // launch: its weight tiles follow the head's through the same ring and one kernel boundary less
+        // lies on the critical path (with per-kernel profiling it stays a launch of its own).
+        proj_done = false;
+        if (h->gemm_impl == 0 && !h->profile && l + 1 < p.n) {
+            GemmCall c[2];
+            c[0].A = S; c[0].B = w.head[l]; c[0].M = rows; c[0].N = w.V; c[0].Kd = w.d_inner;
+            c[0].block_n = p.lay.block_n[l];
+            c[0].epi = GemmEpilogue{};
+            c[0].epi.mode = 1;
+            c[0].epi.part_val = part_val; c[0].epi.part_idx = part_idx; c[0].epi.part_ms = part_ms;
+            c[0].epi.topk = topk[l];
+            c[1] = proj_call(l + 1);
+            rc = launch_gemm_tc_jobs(c, 2, err, st);
+            proj_done = true;
+        } else {
+            rc = run_head_partials(h, S, w.head[l], rows, p.lay.block_n[l], topk[l], part_val, part_idx, part_ms,
+                                   logits_scratch, err, st);
+        }
         if (rc != SPEC_OK) return rc;
         SPEC_PROF_MARK();
         // fold the partials, branch: children (token, cumulative score) of every node

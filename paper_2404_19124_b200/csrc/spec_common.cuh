@@ -102,6 +102,13 @@ struct GemmEpilogue {
 int choose_block_n(int M, int N, int num_sm, bool tensor_bound_pref);
 int launch_gemm_tc(const void *A, const void *B, int M, int N, int Kd, int block_n, const GemmEpilogue &epi,
                    int32_t *err, cudaStream_t st);
+// Up to two contractions in one launch; neither may read what the other writes.
+struct GemmCall {
+    const void *A, *B;
+    int M, N, Kd, block_n;
+    GemmEpilogue epi;
+};
+int launch_gemm_tc_jobs(const GemmCall *calls, int n_calls, int32_t *err, cudaStream_t st);
 
 // ---- debug CUDA-core GEMM (gemm_simt.cu) ------------------------------------------------
 int launch_gemm_simt(const void *A, const void *B, int M, int N, int Kd, float *C, int ldc, cudaStream_t st);
