@@ -29,6 +29,19 @@ __global__ void __launch_bounds__(kRowThreads, 2) mix_ln_gelu_kernel(MixArgs m, 
     }
 }
 
+// The same for levels with more nodes than one wave of the kernel above holds: one 8-element group in
+// flight per thread and at most 80 registers, so three CTAs share an SM and the level stays one wave.
+__global__ void __launch_bounds__(kRowThreads, 3) mix_ln_gelu_many_kernel(MixArgs m, int warm_ctas) {
+    __shared__ float red[32];
+    griddep_launch();
+#pragma unroll 1
+    for (int pass = (int)blockIdx.x < warm_ctas ? 0 : 1; pass < 2; ++pass) {
+        if (pass == 1) griddep_wait();
+        if (m.d <= 8 * kRowThreads) mix_ln_gelu_row<kRowThreads, 1, 1, BlockSync>(m, blockIdx.x, threadIdx.x, red, pass == 1);
+        else mix_ln_gelu_row<kRowThreads, 2, 1, BlockSync>(m, blockIdx.x, threadIdx.x, red, pass == 1);
+    }
+}
+
 // Rows of up to 16384 elements.
 __global__ void __launch_bounds__(kRowThreads) mix_ln_gelu_mid_kernel(MixArgs m, int warm_ctas) {
     __shared__ float red[32];
@@ -107,7 +120,9 @@ int launch_mix_ln_gelu(const float *P, int p_splits, size_t p_split_stride, cons
     m.emb = (const uint16_t *)emb; m.tok = tok; m.gamma = gamma; m.beta = beta;
     m.d = d_inner; m.V = V; m.parent_div = parent_div; m.a = a; m.b = b; m.eps = eps;
     m.S_out = (uint16_t *)S_out; m.err = err;
-    if (d_inner <= 8 * kRowThreads * 2) {
+    if (d_inner <= 8 * kRowThreads * 2 && rows > num_sms()) {
+        SPEC_CUDA_TRY(launch_pdl(mix_ln_gelu_many_kernel, dim3(rows), dim3(kRowThreads), 0, st, m, num_sms()));
+    } else if (d_inner <= 8 * kRowThreads * 2) {
         SPEC_CUDA_TRY(launch_pdl(mix_ln_gelu_kernel, dim3(rows), dim3(kRowThreads), 0, st, m, 2 * num_sms()));
     } else if (d_inner <= 8 * kRowThreads * 8) {
         SPEC_CUDA_TRY(launch_pdl(mix_ln_gelu_mid_kernel, dim3(rows), dim3(kRowThreads), 0, st, m, num_sms()));
