@@ -2,10 +2,8 @@
 //   mix_ln_gelu_kernel   one CTA of 256 threads per tree node
 //   merge_expand_kernel  one CTA of 128 threads per row of the vocabulary head
 //   prune_kernel         one CTA of 256 threads per sequence
-// Each is launched with programmatic stream serialization, so its CTAs are usually resident while the
-// kernel before it still runs.  The CTAs of the first wave (`warm_ctas`) use that wait: they run their
-// step once "dry" (same instructions, no dependent loads, no stores), which brings the code into the
-// SM's instruction cache, then wait for the preceding grid and run it for real.
+// Each is launched with programmatic stream serialization, so its CTAs are usually resident, waiting,
+// while the kernel before it still runs.
 #include "row_ops.cuh"
 
 namespace spec {
@@ -18,40 +16,31 @@ constexpr int kRowThreads = 256;
 constexpr int kMergeThreads = 128;
 
 // Rows of up to 4096 elements: at most 128 registers, so that two CTAs fit beside a resident GEMM CTA.
-__global__ void __launch_bounds__(kRowThreads, 2) mix_ln_gelu_kernel(MixArgs m, int warm_ctas) {
+__global__ void __launch_bounds__(kRowThreads, 2) mix_ln_gelu_kernel(MixArgs m) {
     __shared__ float red[32];
     griddep_launch();
-#pragma unroll 1
-    for (int pass = (int)blockIdx.x < warm_ctas ? 0 : 1; pass < 2; ++pass) {   // one copy of the code, run twice
-        if (pass == 1) griddep_wait();
-        if (m.d <= 8 * kRowThreads) mix_ln_gelu_row<kRowThreads, 1, 2, BlockSync>(m, blockIdx.x, threadIdx.x, red, pass == 1);
-        else mix_ln_gelu_row<kRowThreads, 2, 2, BlockSync>(m, blockIdx.x, threadIdx.x, red, pass == 1);
-    }
+    griddep_wait();
+    if (m.d <= 8 * kRowThreads) mix_ln_gelu_row<kRowThreads, 1, 2, BlockSync>(m, blockIdx.x, threadIdx.x, red);
+    else mix_ln_gelu_row<kRowThreads, 2, 2, BlockSync>(m, blockIdx.x, threadIdx.x, red);
 }
 
 // The same for levels with more nodes than one wave of the kernel above holds: one 8-element group in
 // flight per thread and at most 80 registers, so three CTAs share an SM and the level stays one wave.
-__global__ void __launch_bounds__(kRowThreads, 3) mix_ln_gelu_many_kernel(MixArgs m, int warm_ctas) {
+__global__ void __launch_bounds__(kRowThreads, 3) mix_ln_gelu_many_kernel(MixArgs m) {
     __shared__ float red[32];
     griddep_launch();
-#pragma unroll 1
-    for (int pass = (int)blockIdx.x < warm_ctas ? 0 : 1; pass < 2; ++pass) {
-        if (pass == 1) griddep_wait();
-        if (m.d <= 8 * kRowThreads) mix_ln_gelu_row<kRowThreads, 1, 1, BlockSync>(m, blockIdx.x, threadIdx.x, red, pass == 1);
-        else mix_ln_gelu_row<kRowThreads, 2, 1, BlockSync>(m, blockIdx.x, threadIdx.x, red, pass == 1);
-    }
+    griddep_wait();
+    if (m.d <= 8 * kRowThreads) mix_ln_gelu_row<kRowThreads, 1, 1, BlockSync>(m, blockIdx.x, threadIdx.x, red);
+    else mix_ln_gelu_row<kRowThreads, 2, 1, BlockSync>(m, blockIdx.x, threadIdx.x, red);
 }
 
 // Rows of up to 16384 elements.
-__global__ void __launch_bounds__(kRowThreads) mix_ln_gelu_mid_kernel(MixArgs m, int warm_ctas) {
+__global__ void __launch_bounds__(kRowThreads) mix_ln_gelu_mid_kernel(MixArgs m) {
     __shared__ float red[32];
     griddep_launch();
-#pragma unroll 1
-    for (int pass = (int)blockIdx.x < warm_ctas ? 0 : 1; pass < 2; ++pass) {
-        if (pass == 1) griddep_wait();
-        if (m.d <= 8 * kRowThreads * 4) mix_ln_gelu_row<kRowThreads, 4, 2, BlockSync>(m, blockIdx.x, threadIdx.x, red, pass == 1);
-        else mix_ln_gelu_row<kRowThreads, 8, 2, BlockSync>(m, blockIdx.x, threadIdx.x, red, pass == 1);
-    }
+    griddep_wait();
+    if (m.d <= 8 * kRowThreads * 4) mix_ln_gelu_row<kRowThreads, 4, 2, BlockSync>(m, blockIdx.x, threadIdx.x, red);
+    else mix_ln_gelu_row<kRowThreads, 8, 2, BlockSync>(m, blockIdx.x, threadIdx.x, red);
 }
 
 // Rows wider than the register version covers: the mixed row is staged in shared memory.
@@ -87,27 +76,20 @@ __global__ void __launch_bounds__(kRowThreads) mix_ln_gelu_wide_kernel(MixArgs m
         m.S_out[(size_t)r * d + i] = (uint16_t)float_to_bf16_bits(gelu_erf((h_s[i] - mean) * rstd * m.gamma[i] + m.beta[i]));
 }
 
-__global__ void __launch_bounds__(kMergeThreads) merge_expand_kernel(MergeArgs g, int warm_ctas) {
+__global__ void __launch_bounds__(kMergeThreads) merge_expand_kernel(MergeArgs g) {
     __shared__ Scratch sc;
     griddep_launch();
-#pragma unroll 1
-    for (int pass = (int)blockIdx.x < warm_ctas ? 0 : 1; pass < 2; ++pass) {
-        if (pass == 1) griddep_wait();
-        merge_expand_row<kMergeThreads, BlockSync>(g, blockIdx.x, threadIdx.x, &sc, pass == 1);
-    }
+    griddep_wait();
+    merge_expand_row<kMergeThreads, BlockSync>(g, blockIdx.x, threadIdx.x, &sc);
 }
 
 __global__ void __launch_bounds__(kRowThreads)
-prune_kernel(const float *leaf_score, PruneArgs pa, int L, int Lpad, int K, int32_t *cand_tok, float *cand_logp,
-             int warm_ctas) {
+prune_kernel(const float *leaf_score, PruneArgs pa, int L, int Lpad, int K, int32_t *cand_tok, float *cand_logp) {
     extern __shared__ LeafKey keys[];   // [Lpad]
     griddep_launch();
-#pragma unroll 1
-    for (int pass = (int)blockIdx.x < warm_ctas ? 0 : 1; pass < 2; ++pass) {
-        if (pass == 1) griddep_wait();
-        prune_sequence<kRowThreads, BlockSync>(leaf_score, pa, L, Lpad, K, cand_tok, cand_logp, blockIdx.x, threadIdx.x,
-                                               keys, pass == 1);
-    }
+    griddep_wait();
+    prune_sequence<kRowThreads, BlockSync>(leaf_score, pa, L, Lpad, K, cand_tok, cand_logp, blockIdx.x, threadIdx.x,
+                                           keys);
 }
 
 }  // namespace
@@ -121,11 +103,11 @@ int launch_mix_ln_gelu(const float *P, int p_splits, size_t p_split_stride, cons
     m.d = d_inner; m.V = V; m.parent_div = parent_div; m.a = a; m.b = b; m.eps = eps;
     m.S_out = (uint16_t *)S_out; m.err = err;
     if (d_inner <= 8 * kRowThreads * 2 && rows > num_sms()) {
-        SPEC_CUDA_TRY(launch_pdl(mix_ln_gelu_many_kernel, dim3(rows), dim3(kRowThreads), 0, st, m, num_sms()));
+        SPEC_CUDA_TRY(launch_pdl(mix_ln_gelu_many_kernel, dim3(rows), dim3(kRowThreads), 0, st, m));
     } else if (d_inner <= 8 * kRowThreads * 2) {
-        SPEC_CUDA_TRY(launch_pdl(mix_ln_gelu_kernel, dim3(rows), dim3(kRowThreads), 0, st, m, 2 * num_sms()));
+        SPEC_CUDA_TRY(launch_pdl(mix_ln_gelu_kernel, dim3(rows), dim3(kRowThreads), 0, st, m));
     } else if (d_inner <= 8 * kRowThreads * 8) {
-        SPEC_CUDA_TRY(launch_pdl(mix_ln_gelu_mid_kernel, dim3(rows), dim3(kRowThreads), 0, st, m, num_sms()));
+        SPEC_CUDA_TRY(launch_pdl(mix_ln_gelu_mid_kernel, dim3(rows), dim3(kRowThreads), 0, st, m));
     } else {
         const size_t smem = sizeof(float) * (size_t)d_inner;
         if (smem > 48 * 1024)
@@ -141,7 +123,7 @@ int launch_merge_expand(const float *part_val, const int32_t *part_idx, const fl
     MergeArgs g{};
     g.part_val = part_val; g.part_idx = part_idx; g.part_ms = part_ms;
     g.n_tiles = n_tiles; g.topk = topk; g.score_in = score_in; g.tok_out = tok_out; g.score_out = score_out;
-    SPEC_CUDA_TRY(launch_pdl(merge_expand_kernel, dim3(rows), dim3(kMergeThreads), 0, st, g, 2 * num_sms()));
+    SPEC_CUDA_TRY(launch_pdl(merge_expand_kernel, dim3(rows), dim3(kMergeThreads), 0, st, g));
     return SPEC_OK;
 }
 
@@ -150,7 +132,7 @@ int launch_prune(const float *leaf_score, const PruneArgs &pa, int B, int L, int
     int Lpad = 2;
     while (Lpad < L) Lpad <<= 1;
     SPEC_CUDA_TRY(launch_pdl(prune_kernel, dim3(B), dim3(kRowThreads), sizeof(LeafKey) * (size_t)Lpad, st, leaf_score, pa,
-                             L, Lpad, K, cand_tok, cand_logp, 2 * num_sms()));
+                             L, Lpad, K, cand_tok, cand_logp));
     return SPEC_OK;
 }
 

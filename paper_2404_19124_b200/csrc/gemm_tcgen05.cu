@@ -65,9 +65,8 @@ gemm_tc_kernel(const __grid_constant__ GemmMaps maps, const __grid_constant__ Ge
     } else {
         AccPos ap{0, 0u};
         bool ok = true;
-        // real tiles only become ready after the producer's wait; the dry pass of the first job comes before it
-        for (int q = 0; ok && q < p.n_jobs; ++q) ok = epilogue_job(pp, p.job[q], ap, q == 0);
         griddep_wait();
+        for (int q = 0; ok && q < p.n_jobs; ++q) ok = epilogue_job(pp, p.job[q], ap);
     }
     pipe_teardown(pp, p.tmem_cols);
 }

@@ -6,12 +6,8 @@
 //                     its top-k tokens and log-probabilities and writes the node's children
 //   prune_sequence    orders one sequence's leaves by (score desc, leaf index asc), keeps K, walks
 //                     back to the root to emit the K n-grams
-// These steps run once per launch on a handful of rows, so what they cost is latency: round trips
-// to L2 / HBM (all loads of a step are issued before the first is used) and, on an SM that has not
-// run the code yet, instruction fetch (about 0.1 us per 128 bytes of code).  Every step therefore
-// takes a `live` flag: with live == false the same instructions run but nothing produced by an earlier
-// kernel is read and nothing is written, which a kernel uses to pull its code into the instruction
-// cache while it still waits for the kernel before it.
+// These steps run once per launch on a handful of rows, so what they cost is latency: every load of a
+// step is issued before the first one is used, and dependent chains are kept short.
 // Buffers that a preceding kernel wrote are read with ld.global.cg, never through the non-coherent path.
 #pragma once
 
@@ -70,12 +66,12 @@ struct MixArgs {
 // t, t + kThreads, ... (kIters of them; d <= 8 * kThreads * kIters, d % 8 == 0).  kDepth of those
 // groups have their loads in flight together (registers against latency).
 template <int kThreads, int kIters, int kDepth, typename Sync>
-__device__ __forceinline__ void mix_ln_gelu_row(const MixArgs &m, int r, int tid, float *red, bool live) {
+__device__ __forceinline__ void mix_ln_gelu_row(const MixArgs &m, int r, int tid, float *red) {
     constexpr int kSp = 4;                                        // partial projections fetched per batch
     constexpr int kGroup = kIters >= 8 ? 1 : (kIters < kDepth ? kIters : kDepth);
-    const int t = live ? __ldcg(m.tok + r) : 0;
+    const int t = __ldcg(m.tok + r);
     const bool tok_ok = (t >= 0) && (t < m.V);
-    if (!tok_ok && tid == 0 && live) report_error(m.err, SPEC_ERR_TOKEN_RANGE);
+    if (!tok_ok && tid == 0) report_error(m.err, SPEC_ERR_TOKEN_RANGE);
     const int d = m.d;
     const float *p = m.P + (size_t)(r / m.parent_div) * d;
     const uint16_t *e = m.emb + (size_t)(tok_ok ? t : 0) * d;
@@ -96,7 +92,7 @@ __device__ __forceinline__ void mix_ln_gelu_row(const MixArgs &m, int r, int tid
             for (int sp = 0; sp < kSp; ++sp) {
                 pa[q][sp] = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
                 pb[q][sp] = pa[q][sp];
-                if (i < d && sp < m.p_splits && live) {
+                if (i < d && sp < m.p_splits) {
                     pa[q][sp] = __ldcg((const float4 *)(p + sp * m.p_split_stride + i));
                     pb[q][sp] = __ldcg((const float4 *)(p + sp * m.p_split_stride + i + 4));
                 }
@@ -112,7 +108,7 @@ __device__ __forceinline__ void mix_ln_gelu_row(const MixArgs &m, int r, int tid
                 pv[0] += pa[q][sp].x; pv[1] += pa[q][sp].y; pv[2] += pa[q][sp].z; pv[3] += pa[q][sp].w;
                 pv[4] += pb[q][sp].x; pv[5] += pb[q][sp].y; pv[6] += pb[q][sp].z; pv[7] += pb[q][sp].w;
             }
-            if (i < d && live) {
+            if (i < d) {
                 for (int sp = kSp; sp < m.p_splits; ++sp) {   // more partials than one batch holds (rare)
                     const float4 p0 = __ldcg((const float4 *)(p + sp * m.p_split_stride + i));
                     const float4 p1 = __ldcg((const float4 *)(p + sp * m.p_split_stride + i + 4));
@@ -180,18 +176,18 @@ __device__ __forceinline__ void mix_ln_gelu_row(const MixArgs &m, int r, int tid
             const float s1 = gelu_erf((h[it][j + 1] - mean) * rstd * gv[j + 1] + bv[j + 1]);
             packed[j >> 1] = float_to_bf16_bits(s0) | (float_to_bf16_bits(s1) << 16);
         }
-        if (i < d && live) *(uint4 *)(m.S_out + (size_t)r * d + i) = make_uint4(packed[0], packed[1], packed[2], packed[3]);
+        if (i < d) *(uint4 *)(m.S_out + (size_t)r * d + i) = make_uint4(packed[0], packed[1], packed[2], packed[3]);
     }
 }
 
 // Picks the register-array size for the row width; false when the row is too wide for this group size.
 template <int kThreads, int kDepth, typename Sync>
-__device__ __forceinline__ bool mix_ln_gelu_row_any(const MixArgs &m, int r, int tid, float *red, bool live) {
+__device__ __forceinline__ bool mix_ln_gelu_row_any(const MixArgs &m, int r, int tid, float *red) {
     const int groups = (m.d + 8 * kThreads - 1) / (8 * kThreads);
-    if (groups <= 1) mix_ln_gelu_row<kThreads, 1, kDepth, Sync>(m, r, tid, red, live);
-    else if (groups <= 2) mix_ln_gelu_row<kThreads, 2, kDepth, Sync>(m, r, tid, red, live);
-    else if (groups <= 4) mix_ln_gelu_row<kThreads, 4, kDepth, Sync>(m, r, tid, red, live);
-    else if (groups <= 8) mix_ln_gelu_row<kThreads, 8, kDepth, Sync>(m, r, tid, red, live);
+    if (groups <= 1) mix_ln_gelu_row<kThreads, 1, kDepth, Sync>(m, r, tid, red);
+    else if (groups <= 2) mix_ln_gelu_row<kThreads, 2, kDepth, Sync>(m, r, tid, red);
+    else if (groups <= 4) mix_ln_gelu_row<kThreads, 4, kDepth, Sync>(m, r, tid, red);
+    else if (groups <= 8) mix_ln_gelu_row<kThreads, 8, kDepth, Sync>(m, r, tid, red);
     else return false;
     return true;
 }
@@ -281,15 +277,15 @@ __device__ __forceinline__ void fold_max_sum(float &m, float &s, const float2 &m
 // best in `topk` rounds; a round is two warp-wide integer reductions (redux.sync: maximum of the value
 // keys, then minimum token id among the lanes that hold it) and one shared-memory exchange between warps.
 template <int kThreads, typename Sync>
-__device__ __forceinline__ void merge_expand_row(const MergeArgs &g, int r, int tid, Scratch *sc, bool live) {
+__device__ __forceinline__ void merge_expand_row(const MergeArgs &g, int r, int tid, Scratch *sc) {
     constexpr int kWarps = kThreads / 32;
     constexpr int kT = SPEC_MAX_TOPK;
     const int lane = tid & 31, warp = tid >> 5;
-    const int n_tiles = live ? g.n_tiles : min(g.n_tiles, 1), topk = g.topk;
+    const int n_tiles = g.n_tiles, topk = g.topk;
     const float4 *pv4 = (const float4 *)(g.part_val + (size_t)r * g.n_tiles * kT);
     const int4 *pi4 = (const int4 *)(g.part_idx + (size_t)r * g.n_tiles * kT);
     const float2 *pms = (const float2 *)(g.part_ms + (size_t)r * g.n_tiles * 2);
-    const float base = (g.score_in && live) ? __ldcg(g.score_in + r) : 0.0f;
+    const float base = (g.score_in) ? __ldcg(g.score_in + r) : 0.0f;
 
     float tv[kT];
     int ti[kT];
@@ -303,16 +299,11 @@ __device__ __forceinline__ void merge_expand_row(const MergeArgs &g, int r, int 
         const int t2 = t + kThreads;
         const bool has2 = t2 < n_tiles;
         const int tb = has2 ? t2 : t;
-        float2 ms_a = make_float2(-INFINITY, 0.0f), ms_b = ms_a;
-        float4 va0 = make_float4(0.f, 0.f, 0.f, 0.f), va1 = va0, vb0 = va0, vb1 = va0;
-        int4 ia0 = make_int4(0, 1, 2, 3), ia1 = make_int4(4, 5, 6, 7), ib0 = ia0, ib1 = ia1;
-        if (live) {
-            ms_a = __ldcg(pms + t); ms_b = __ldcg(pms + tb);
-            va0 = __ldcg(pv4 + 2 * t); va1 = __ldcg(pv4 + 2 * t + 1);
-            ia0 = __ldcg(pi4 + 2 * t); ia1 = __ldcg(pi4 + 2 * t + 1);
-            vb0 = __ldcg(pv4 + 2 * tb); vb1 = __ldcg(pv4 + 2 * tb + 1);
-            ib0 = __ldcg(pi4 + 2 * tb); ib1 = __ldcg(pi4 + 2 * tb + 1);
-        }
+        const float2 ms_a = __ldcg(pms + t), ms_b = __ldcg(pms + tb);
+        const float4 va0 = __ldcg(pv4 + 2 * t), va1 = __ldcg(pv4 + 2 * t + 1);
+        const int4 ia0 = __ldcg(pi4 + 2 * t), ia1 = __ldcg(pi4 + 2 * t + 1);
+        const float4 vb0 = __ldcg(pv4 + 2 * tb), vb1 = __ldcg(pv4 + 2 * tb + 1);
+        const int4 ib0 = __ldcg(pi4 + 2 * tb), ib1 = __ldcg(pi4 + 2 * tb + 1);
         fold_max_sum(m, s, ms_a);
         if (has2) fold_max_sum(m, s, ms_b);
         fold_tile_list(tv, ti, va0, va1, ia0, ia1, topk, true);
@@ -369,7 +360,7 @@ __device__ __forceinline__ void merge_expand_row(const MergeArgs &g, int r, int 
             tv[kT - 1] = -INFINITY;
             ti[kT - 1] = 0x7fffffff;
         }
-        if (tid == 0 && live) {
+        if (tid == 0) {
             g.tok_out[(size_t)r * topk + j] = bi;
             g.score_out[(size_t)r * topk + j] = base + (key_float(bk) - lse);
         }
@@ -387,12 +378,12 @@ __device__ __forceinline__ bool leaf_before(const LeafKey &a, const LeafKey &b) 
 
 // Writes candidate `rank` of sequence b: its score and the tokens on the path from the root to `leaf`.
 __device__ __forceinline__ void emit_candidate(const PruneArgs &pa, int L, int K, int32_t *cand_tok, float *cand_logp,
-                                               int b, int rank, float score, int leaf, bool live) {
-    if (live) cand_logp[(size_t)b * K + rank] = score;
+                                               int b, int rank, float score, int leaf) {
+    cand_logp[(size_t)b * K + rank] = score;
     int idx = leaf;            // index among this sequence's nodes of level n
     int per_seq = L;           // nodes of this sequence at level l + 1
     for (int l = pa.n - 1; l >= 0; --l) {
-        if (live) cand_tok[((size_t)b * K + rank) * pa.n + l] = __ldcg(pa.tok[l] + (size_t)b * per_seq + idx);
+        cand_tok[((size_t)b * K + rank) * pa.n + l] = __ldcg(pa.tok[l] + (size_t)b * per_seq + idx);
         idx /= pa.topk[l];
         per_seq /= pa.topk[l];
     }
@@ -404,11 +395,10 @@ __device__ __forceinline__ void emit_candidate(const PruneArgs &pa, int L, int K
 // bitonically.
 template <int kThreads, typename Sync>
 __device__ __forceinline__ void prune_sequence(const float *leaf_score, const PruneArgs &pa, int L, int Lpad, int K,
-                                               int32_t *cand_tok, float *cand_logp, int b, int tid, LeafKey *keys,
-                                               bool live) {
+                                               int32_t *cand_tok, float *cand_logp, int b, int tid, LeafKey *keys) {
     Sync::sync();   // a previous call may still be reading the keys
     for (int i = tid; i < Lpad; i += kThreads) {
-        keys[i].score = (i < L && live) ? __ldcg(leaf_score + (size_t)b * L + i) : -INFINITY;
+        keys[i].score = (i < L) ? __ldcg(leaf_score + (size_t)b * L + i) : -INFINITY;
         keys[i].leaf = i < L ? i : 0x7fffffff;
     }
     Sync::sync();
@@ -417,7 +407,7 @@ __device__ __forceinline__ void prune_sequence(const float *leaf_score, const Pr
             const LeafKey mine = keys[i];
             int rank = 0;
             for (int j = 0; j < L; ++j) rank += leaf_before(keys[j], mine) ? 1 : 0;
-            if (rank < K) emit_candidate(pa, L, K, cand_tok, cand_logp, b, rank, mine.score, mine.leaf, live);
+            if (rank < K) emit_candidate(pa, L, K, cand_tok, cand_logp, b, rank, mine.score, mine.leaf);
         }
         return;
     }
@@ -438,7 +428,7 @@ __device__ __forceinline__ void prune_sequence(const float *leaf_score, const Pr
         }
     }
     for (int k = tid; k < K; k += kThreads)
-        emit_candidate(pa, L, K, cand_tok, cand_logp, b, k, keys[k].score, keys[k].leaf, live);
+        emit_candidate(pa, L, K, cand_tok, cand_logp, b, k, keys[k].score, keys[k].leaf);
 }
 
 }  // namespace rows

@@ -448,30 +448,20 @@ __device__ __forceinline__ void epilogue_topk(const GemmJob &p, uint32_t taddr, 
 }
 
 // ---- epilogue warps (warps 2-5, all lanes) ----------------------------------------------------------
-// `warm`: before the first tile the loop body runs once "dry" on whatever the accumulator slot holds,
-// with every row marked invalid so that nothing is stored and no barrier is touched.  The epilogue
-// code (tens of KB when unrolled) is then in the SM's instruction cache when the first real tile, whose
-// epilogue nothing overlaps in a one-tile-per-CTA launch, arrives; the warps would only idle otherwise.
-__device__ __forceinline__ bool epilogue_job(const Pipe &pp, const GemmJob &j, AccPos &ap, bool warm) {
+__device__ __forceinline__ bool epilogue_job(const Pipe &pp, const GemmJob &j, AccPos &ap) {
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int quarter = warp & 3;               // TMEM lane quarter this warp may read
     const int row_in_tile = quarter * 32 + lane;
     const int mn_tiles = j.m_tiles * j.n_tiles;
     const int num_tiles = mn_tiles * j.splits;
     Barriers *bars = pp.bars;
-    const int first = first_tile_of(j);
-    if (first >= num_tiles) return true;
-    bool dry = warm;
-#pragma unroll 1
-    for (int tile = first; tile < num_tiles; tile += dry ? 0 : (int)gridDim.x, dry = false) {
+    for (int tile = first_tile_of(j); tile < num_tiles; tile += gridDim.x) {
         const int split = tile / mn_tiles, mn = tile - split * mn_tiles;
         const int m_tile = mn % j.m_tiles, n_tile = mn / j.m_tiles;
-        if (!dry) {
-            if (!mbar_wait(&bars->acc_full[ap.acc], ap.phase, bars, pp.err)) return false;
-            tc_fence_after();
-        }
+        if (!mbar_wait(&bars->acc_full[ap.acc], ap.phase, bars, pp.err)) return false;
+        tc_fence_after();
         const int row = m_tile * kBlockM + row_in_tile;
-        const bool row_ok = row < j.M && !dry;
+        const bool row_ok = row < j.M;
         const uint32_t taddr = pp.tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(ap.acc * pp.acc_stride);
         const int col0 = n_tile * j.block_n;
         if (j.epi.mode == 0) {
@@ -510,7 +500,6 @@ __device__ __forceinline__ bool epilogue_job(const Pipe &pp, const GemmJob &j, A
             if (j.epi.topk <= 4) epilogue_topk<4>(j, taddr, row, row_ok, col0, n_tile);
             else epilogue_topk<SPEC_MAX_TOPK>(j, taddr, row, row_ok, col0, n_tile);
         }
-        if (dry) continue;
         tc_fence_before();
         __syncwarp();
         if (lane == 0) mbar_arrive(&bars->acc_empty[ap.acc]);
