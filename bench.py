@@ -348,6 +348,16 @@ def main():
     v1.record(stream)
     torch.cuda.synchronize()
     verify_ms = v0.elapsed_time(v1) / prof_steps
+    # the early-exit form on the same inputs (reads only the rows up to each candidate's first mismatch)
+    for i in range(3):
+        B.spec_verify(cand, rot[i % n_rot], accept_len=acc, best_cand=best, next_tok=nxt, workspace=vws, early_exit=True)
+    torch.cuda.synchronize()
+    v0.record(stream)
+    for i in range(prof_steps):
+        B.spec_verify(cand, rot[i % n_rot], accept_len=acc, best_cand=best, next_tok=nxt, workspace=vws, early_exit=True)
+    v1.record(stream)
+    torch.cuda.synchronize()
+    verify_early_ms = v0.elapsed_time(v1) / prof_steps
 
     # the vocabulary head alone at M = B*K rows (GEMM + merge kernels back to back), last head's weights
     bk_rows = Bn * K
@@ -396,7 +406,8 @@ def main():
     v_gbs = logits_bytes / (verify_ms * 1e-3) / 1e9
     roof_verify = {"kernel": "verify_stream_kernel + verify_accept_kernel", "bound": "hbm", "achieved": v_gbs,
                    "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": v_gbs / peaks["hbm_gbs"], "traffic": None,
-                   "us": round(verify_ms * 1e3, 2), "bytes": logits_bytes}
+                   "us": round(verify_ms * 1e3, 2), "bytes": logits_bytes,
+                   "early_exit_form_us": round(verify_early_ms * 1e3, 2)}
     # heads below the ridge are weight-bandwidth bound: report their HBM fraction too
     head_hbm = {}
     for l in range(n):

@@ -134,6 +134,18 @@ int spec_verify(const int32_t *cand_tok, const void *base_logits, int logits_dty
                 int32_t *accept_len, int32_t *best_cand, int32_t *next_tok, void *workspace,
                 size_t workspace_bytes, void *cuda_stream);
 
+/* Early-exit form of spec_verify (Sec. 1: everything after a candidate's first rejected token is
+ * discarded, so the base model's logits behind it need not be looked at).  Same arguments, same
+ * three results.  One thread block per candidate reads its rows in order and stops after the first
+ * row whose arg-max differs from the speculated token: the bytes read fall from B K (n+1) V elements
+ * to sum over the candidates of (m[b,k] + 1) V.  In the workspace, g holds -1 for rows that were not
+ * read.  Worth it when many candidates fail early or the tensor is large; when nearly all rows are
+ * needed the one-pass streaming form is faster.  Rows must be whole 16-byte vectors and base_logits
+ * 16-byte aligned, otherwise the call silently runs the streaming form. */
+int spec_verify_early(const int32_t *cand_tok, const void *base_logits, int logits_dtype, int B, int K, int n, int V,
+                      int32_t *accept_len, int32_t *best_cand, int32_t *next_tok, void *workspace,
+                      size_t workspace_bytes, void *cuda_stream);
+
 /* ---- verify without a caller-supplied workspace -----------------------------------------
  * (No counterpart in the paper: this is a packaging variant of spec_verify, same results.)
  * Some hosts of this library cannot hand it scratch memory: a serving process that gave all

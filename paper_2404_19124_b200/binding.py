@@ -26,7 +26,7 @@ EXPORTS = [
     "spec_version", "spec_status_str", "spec_last_cuda_error", "spec_create", "spec_destroy", "spec_set_option",
     "spec_draft_workspace_bytes", "spec_draft_layout", "spec_draft", "spec_verify_workspace_bytes", "spec_verify",
     "spec_profile_read", "spec_poll_error", "spec_head_workspace_bytes", "spec_head_logits", "spec_head_topk",
-    "spec_verify_static",
+    "spec_verify_static", "spec_verify_early",
 ]
 
 if not os.path.exists(LIB_PATH):
@@ -75,6 +75,7 @@ _lib.spec_verify.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_int, 
                              C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]
 _lib.spec_verify_static.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_int, C.c_int, C.c_int,
                                     C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
+_lib.spec_verify_early.argtypes = _lib.spec_verify.argtypes
 _lib.spec_poll_error.argtypes = [C.c_void_p, C.c_void_p]
 _lib.spec_profile_read.argtypes = [C.c_void_p, C.POINTER(C.c_float), C.c_int, C.POINTER(C.c_int)]
 _lib.spec_head_workspace_bytes.restype = C.c_size_t
@@ -226,8 +227,10 @@ def spec_verify_workspace_bytes(B: int, K: int, n: int, V: int, logits_dtype: in
 
 def spec_verify(cand_tok: torch.Tensor, base_logits: torch.Tensor, accept_len: Optional[torch.Tensor] = None,
                 best_cand: Optional[torch.Tensor] = None, next_tok: Optional[torch.Tensor] = None,
-                workspace: Optional[torch.Tensor] = None, stream: Optional[torch.cuda.Stream] = None):
-    """Enqueues one verification; returns (accept_len, best_cand, next_tok, workspace), int32 [B] each."""
+                workspace: Optional[torch.Tensor] = None, stream: Optional[torch.cuda.Stream] = None,
+                early_exit: bool = False):
+    """Enqueues one verification; returns (accept_len, best_cand, next_tok, workspace), int32 [B] each.
+    early_exit: the form that stops reading a candidate's rows at its first mismatch (spec_verify_early)."""
     B, K, n = cand_tok.shape
     _dev(cand_tok, torch.int32, name="cand_tok")
     if base_logits.dtype == torch.bfloat16:
@@ -249,8 +252,9 @@ def spec_verify(cand_tok: torch.Tensor, base_logits: torch.Tensor, accept_len: O
         if need == 0:
             raise SpecError(SPEC_ERR_SHAPE, "spec_verify_workspace_bytes")
         workspace = torch.empty(need, dtype=torch.uint8, device=dev)
-    _check(_lib.spec_verify(_ptr(cand_tok), _ptr(base_logits), dt, B, K, n, V, _ptr(outs[0]), _ptr(outs[1]),
-                            _ptr(outs[2]), _ptr(workspace), workspace.numel(), _stream_ptr(stream)), "spec_verify")
+    fn = _lib.spec_verify_early if early_exit else _lib.spec_verify
+    _check(fn(_ptr(cand_tok), _ptr(base_logits), dt, B, K, n, V, _ptr(outs[0]), _ptr(outs[1]),
+              _ptr(outs[2]), _ptr(workspace), workspace.numel(), _stream_ptr(stream)), "spec_verify")
     return outs[0], outs[1], outs[2], workspace
 
 

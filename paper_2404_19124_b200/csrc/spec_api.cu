@@ -433,6 +433,27 @@ int spec_verify(const int32_t *cand_tok, const void *base_logits, int logits_dty
                          plan, (cudaStream_t)cuda_stream);
 }
 
+int spec_verify_early(const int32_t *cand_tok, const void *base_logits, int logits_dtype, int B, int K, int n, int V,
+                      int32_t *accept_len, int32_t *best_cand, int32_t *next_tok, void *workspace,
+                      size_t workspace_bytes, void *cuda_stream) {
+    if (!cand_tok || !base_logits || !accept_len || !best_cand || !next_tok) return SPEC_ERR_INVALID_ARG;
+    if (B <= 0 || K <= 0 || n <= 0 || V <= 0) return SPEC_ERR_INVALID_ARG;
+    if (logits_dtype != SPEC_BF16 && logits_dtype != SPEC_F32) return SPEC_ERR_INVALID_ARG;
+    if (K > 65535 || (long long)K * (n + 1) > 12288 || n > 32767) return SPEC_ERR_SHAPE;
+    if ((long long)B * K * (n + 1) > (1ll << 30)) return SPEC_ERR_SHAPE;
+    if (((uintptr_t)base_logits % (logits_dtype == SPEC_BF16 ? 2 : 4)) != 0) return SPEC_ERR_INVALID_ARG;
+    const VerifyPlan plan = make_verify_plan(B, K, n, V, logits_dtype);
+    if (!workspace || ((uintptr_t)workspace % kWsAlign) != 0 || workspace_bytes < plan.total)
+        return SPEC_ERR_WORKSPACE;
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    const int rc = launch_verify_early(cand_tok, base_logits, logits_dtype, B, K, n, V, accept_len, best_cand, next_tok,
+                                       workspace, plan, st);
+    if (rc != SPEC_ERR_SHAPE) return rc;
+    // rows that are not whole 16-byte vectors: the streaming form reads everything
+    return launch_verify(cand_tok, base_logits, logits_dtype, B, K, n, V, accept_len, best_cand, next_tok, workspace,
+                         plan, st);
+}
+
 int spec_poll_error(void *workspace, void *cuda_stream) {
     if (!workspace) return SPEC_ERR_INVALID_ARG;
     cudaStream_t st = (cudaStream_t)cuda_stream;

@@ -85,6 +85,10 @@ int launch_verify(const int32_t *cand_tok, const void *base_logits, int dtype, i
                   int32_t *accept_len, int32_t *best_cand, int32_t *next_tok, void *ws, const VerifyPlan &plan,
                   cudaStream_t st);
 
+int launch_verify_early(const int32_t *cand_tok, const void *base_logits, int dtype, int B, int K, int n, int V,
+                        int32_t *accept_len, int32_t *best_cand, int32_t *next_tok, void *ws, const VerifyPlan &plan,
+                        cudaStream_t st);
+
 // ---- tensor-core GEMM (gemm_tcgen05.cu) -------------------------------------------------
 // C[M, N] = A[M, Kd] * B[N, Kd]^T, A and B bf16 row-major (K-major), fp32 accumulation in TMEM.
 struct GemmEpilogue {

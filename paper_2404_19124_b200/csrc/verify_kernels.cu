@@ -234,6 +234,98 @@ verify_accept_kernel(const int32_t *__restrict__ cand_tok, const float *__restri
     }
 }
 
+// ---- early-exit form ------------------------------------------------------------------------------
+// The rows of a candidate matter only up to its first mismatch (Sec. 1: the tokens after a rejected
+// one are discarded), so reading them is optional work: one CTA per candidate walks its rows in order,
+// takes the arg-max of a row with the whole CTA (eight 128-bit loads in flight per thread) and stops
+// after the first row whose arg-max differs from the speculated token.  Bytes read fall from
+// B K (n+1) V to sum over candidates of (m + 1) V elements; rows that were not read get g = -1.
+template <bool kBf16>
+__global__ void __launch_bounds__(kArgmaxThreads)
+verify_early_kernel(const uint4 *__restrict__ logits, const int32_t *__restrict__ cand_tok, int n, int vpr,
+                    int32_t *__restrict__ g, int32_t *__restrict__ match_len) {
+    __shared__ float s_val[kWarpsPerBlock];
+    __shared__ int s_idx[kWarpsPerBlock];
+    __shared__ int s_arg;
+    griddep_launch();
+    griddep_wait();
+    constexpr int kEpv = kBf16 ? 8 : 4;
+    const int c = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    int m = n, j = 0;
+    for (; j <= n; ++j) {
+        const uint4 *rp = logits + ((size_t)c * (n + 1) + j) * vpr;
+        float best = -INFINITY;
+        int idx = kIdxNone;
+        for (int p0 = tid; p0 < vpr; p0 += kArgmaxThreads * kStreamUnroll) {
+            uint4 q[kStreamUnroll];
+#pragma unroll
+            for (int u = 0; u < kStreamUnroll; ++u)
+                if (p0 + kArgmaxThreads * u < vpr) q[u] = ld_stream(rp + p0 + kArgmaxThreads * u);
+#pragma unroll
+            for (int u = 0; u < kStreamUnroll; ++u) {
+                if (p0 + kArgmaxThreads * u < vpr) {
+                    const int base = (p0 + kArgmaxThreads * u) * kEpv;
+                    if (kBf16) consume_bf16(q[u], base, best, idx);
+                    else consume_f32(q[u], base, best, idx);
+                }
+            }
+        }
+        warp_argmax(best, idx);
+        if (lane == 0) {
+            s_val[warp] = best;
+            s_idx[warp] = idx;
+        }
+        __syncthreads();
+        if (tid == 0) {
+            float bv = -INFINITY;
+            int arg = 0;   // a row without any value above -inf (all NaN) yields 0
+            int bi = kIdxNone;
+            for (int w = 0; w < kWarpsPerBlock; ++w) {
+                if (s_val[w] > bv || (s_val[w] == bv && s_idx[w] < bi)) {   // the lowest index among equal maxima
+                    bv = s_val[w];
+                    bi = s_idx[w];
+                }
+            }
+            if (bi != kIdxNone && bv > -INFINITY) arg = bi;
+            s_arg = arg;
+            g[(size_t)c * (n + 1) + j] = arg;
+        }
+        __syncthreads();
+        const int arg = s_arg;
+        if (j < n && cand_tok[(size_t)c * n + j] != arg) {   // uniform over the CTA
+            m = j;
+            break;
+        }
+    }
+    for (int jj = j + 1 + tid; jj <= n; jj += kArgmaxThreads) g[(size_t)c * (n + 1) + jj] = -1;
+    if (tid == 0) match_len[c] = m;
+}
+
+// One CTA per sequence: the candidate with the longest match (lowest index among equals) and its bonus token.
+__global__ void __launch_bounds__(128)
+verify_accept_early_kernel(const int32_t *__restrict__ g, const int32_t *__restrict__ match_len, int K, int n,
+                           int32_t *__restrict__ accept_len, int32_t *__restrict__ best_cand,
+                           int32_t *__restrict__ next_tok, int32_t *err) {
+    __shared__ unsigned int key_s;
+    griddep_launch();
+    griddep_wait();
+    const int b = blockIdx.x;
+    if (threadIdx.x == 0) {
+        key_s = 0u;
+        if (b == 0 && err != nullptr) *err = 0;
+    }
+    __syncthreads();
+    for (int k = threadIdx.x; k < K; k += blockDim.x)
+        atomicMax(&key_s, ((unsigned)match_len[(size_t)b * K + k] << 16) | (unsigned)(0xffff - k));
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        const int m = (int)(key_s >> 16), k = 0xffff - (int)(key_s & 0xffffu);
+        accept_len[b] = m;
+        best_cand[b] = k;
+        next_tok[b] = g[((size_t)b * K + k) * (n + 1) + m];
+    }
+}
+
 size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 }  // namespace
@@ -317,6 +409,28 @@ int launch_verify(const int32_t *cand_tok, const void *base_logits, int dtype, i
     SPEC_CUDA_TRY(launch_pdl(verify_accept_kernel, dim3(B), dim3(128), smem, st, cand_tok, (const float *)pval,
                              (const int32_t *)pidx, K, n, stream ? plan.slots : plan.chunks, plan.vpr, vec_per_warp,
                              g, accept_len, best_cand, next_tok, err));
+    return SPEC_OK;
+}
+
+// Early-exit form; returns SPEC_ERR_SHAPE when the rows are not whole 16-byte vectors (the caller then
+// uses the streaming form).
+int launch_verify_early(const int32_t *cand_tok, const void *base_logits, int dtype, int B, int K, int n, int V,
+                        int32_t *accept_len, int32_t *best_cand, int32_t *next_tok, void *ws, const VerifyPlan &plan,
+                        cudaStream_t st) {
+    if (plan.vpr <= 0 || ((uintptr_t)base_logits % 16) != 0) return SPEC_ERR_SHAPE;
+    char *w = (char *)ws;
+    int32_t *err = (int32_t *)w;
+    int32_t *g = (int32_t *)(w + plan.off_g);
+    int32_t *match_len = (int32_t *)(w + plan.off_pval);   // B * K words; the partial-maxima area is not used here
+    const uint4 *lp = (const uint4 *)base_logits;
+    if (dtype == SPEC_BF16)
+        SPEC_CUDA_TRY(launch_pdl(verify_early_kernel<true>, dim3(B * K), dim3(kArgmaxThreads), 0, st, lp, cand_tok, n,
+                                 plan.vpr, g, match_len));
+    else
+        SPEC_CUDA_TRY(launch_pdl(verify_early_kernel<false>, dim3(B * K), dim3(kArgmaxThreads), 0, st, lp, cand_tok, n,
+                                 plan.vpr, g, match_len));
+    SPEC_CUDA_TRY(launch_pdl(verify_accept_early_kernel, dim3(B), dim3(128), 0, st, (const int32_t *)g,
+                             (const int32_t *)match_len, K, n, accept_len, best_cand, next_tok, err));
     return SPEC_OK;
 }
 

@@ -24,17 +24,35 @@ def _np_logits(x: torch.Tensor):
     return x.detach().cpu().numpy(), oracle.F32
 
 
-def _run_and_compare(B, cand: torch.Tensor, logits: torch.Tensor):
+def _check_g(g_gpu, o_g, cand_np, early):
+    """Streaming form: every row's arg-max.  Early-exit form: rows up to and including a candidate's
+    first mismatch (all n + 1 rows when everything matches) equal the oracle's, the rest hold -1."""
+    if not early:
+        assert np.array_equal(g_gpu, o_g)
+        return
+    Bn, K, n = cand_np.shape
+    m = np.zeros((Bn, K), np.int64)
+    for j in range(n - 1, -1, -1):
+        m = np.where(cand_np[:, :, j] == o_g[:, :, j], m + 1, 0)     # matched prefix length
+    read = np.arange(n + 1)[None, None, :] <= m[:, :, None]
+    assert np.array_equal(g_gpu[read], o_g[read])
+    assert (g_gpu[~read] == -1).all()
+
+
+def _run_and_compare(B, cand: torch.Tensor, logits: torch.Tensor, forms=(False, True)):
     Bn, K, n = cand.shape
-    acc, best, nxt, ws = B.spec_verify(cand.cuda(), logits.cuda())
-    assert B.spec_poll_error(ws) == 0
-    g_gpu = ws_view(ws, 256, Bn * K * (n + 1), torch.int32).cpu().numpy().reshape(Bn, K, n + 1)
     ln, dt = _np_logits(logits)
     o_acc, o_best, o_nxt, o_g = oracle.verify(cand.cpu().numpy(), ln, dt, want_g=True)
-    assert np.array_equal(g_gpu, o_g)
-    assert np.array_equal(acc.cpu().numpy(), o_acc)
-    assert np.array_equal(best.cpu().numpy(), o_best)
-    assert np.array_equal(nxt.cpu().numpy(), o_nxt)
+    for early in forms:
+        acc, best, nxt, ws = B.spec_verify(cand.cuda(), logits.cuda(), early_exit=early)
+        assert B.spec_poll_error(ws) == 0
+        g_gpu = ws_view(ws, 256, Bn * K * (n + 1), torch.int32).cpu().numpy().reshape(Bn, K, n + 1)
+        V = logits.shape[-1]
+        vectors = V % (8 if logits.dtype == torch.bfloat16 else 4) == 0     # else the early form falls back
+        _check_g(g_gpu, o_g, cand.cpu().numpy(), early and vectors)
+        assert np.array_equal(acc.cpu().numpy(), o_acc)
+        assert np.array_equal(best.cpu().numpy(), o_best)
+        assert np.array_equal(nxt.cpu().numpy(), o_nxt)
     return o_acc
 
 
@@ -105,22 +123,26 @@ def test_verify_worked_example(B):
 
 @pytest.mark.parametrize("name", ["tiny", "llama2-7b", "llama2-13b", "codellama-34b", "llama3-8b"])
 def test_verify_full_size_configs(B, name):
-    """Full BASELINE shapes in the launch configuration the benchmark times; the oracle
-    checks every row (the CPU arg-max over the whole tensor takes seconds)."""
+    """Full BASELINE shapes in the launch configuration the benchmark times, streaming and early-exit
+    forms; the oracle checks every row (the CPU arg-max over the whole tensor takes seconds)."""
     cfg = synth.CONFIGS[name]
     cand = synth.random_cand_tok(cfg, device="cuda")
     logits = synth.make_base_logits(cfg, cand, device="cuda")
-    acc, best, nxt, ws = B.spec_verify(cand, logits)
-    torch.cuda.synchronize()
     rows = cfg.B * cfg.K * (cfg.n + 1)
-    g_gpu = ws_view(ws, 256, rows, torch.int32).cpu().numpy().reshape(cfg.B, cfg.K, cfg.n + 1)
+    got = []
+    for early in (False, True):
+        acc, best, nxt, ws = B.spec_verify(cand, logits, early_exit=early)
+        torch.cuda.synchronize()
+        g_gpu = ws_view(ws, 256, rows, torch.int32).cpu().numpy().reshape(cfg.B, cfg.K, cfg.n + 1)
+        got.append((g_gpu, acc.cpu().numpy(), best.cpu().numpy(), nxt.cpu().numpy()))
     bits = synth.bf16_bits(logits)
     del logits
     o_acc, o_best, o_nxt, o_g = oracle.verify(cand.cpu().numpy(), bits, oracle.BF16, want_g=True)
-    assert np.array_equal(g_gpu, o_g)
-    assert np.array_equal(acc.cpu().numpy(), o_acc)
-    assert np.array_equal(best.cpu().numpy(), o_best)
-    assert np.array_equal(nxt.cpu().numpy(), o_nxt)
+    for early, (g_gpu, acc, best, nxt) in zip((False, True), got):
+        _check_g(g_gpu, o_g, cand.cpu().numpy(), early)
+        assert np.array_equal(acc, o_acc)
+        assert np.array_equal(best, o_best)
+        assert np.array_equal(nxt, o_nxt)
     if cfg.plant != "none":
         assert o_acc.max() >= 1
 
