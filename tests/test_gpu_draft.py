@@ -118,10 +118,22 @@ def test_head_topk_exact_ties_prefer_lower_token_id(B):
     B.spec_destroy(h)
 
 
-def _draft_and_check(B, cfg, seqs=None, impl=0, check_levels=False):
+def _draft_and_check(B, cfg, seqs=None, impl=0, check_levels=False, tie_weights=False):
     """Runs spec_draft at the config's full batch and compares the sequences in `seqs`
-    (default: all) with the oracle, one sequence at a time (sequences are independent)."""
-    sw, ow, gw = _setup(cfg)
+    (default: all) with the oracle, one sequence at a time (sequences are independent).
+    tie_weights: every head after the first aliases the second head's tensors (the weight-tied
+    variant the paper mentions in Sec. 3.1 / Sec. 5: same computation, shared parameters)."""
+    if tie_weights:
+        sw = synth.make_weights(cfg)
+        for l in range(2, cfg.n):
+            for lst in (sw.emb, sw.proj, sw.ln_gamma, sw.ln_beta, sw.head):
+                lst[l] = lst[1]
+        ow, gw = to_oracle_weights(sw), weights_to_cuda(sw)
+        for l in range(2, cfg.n):       # on the device too the heads share one copy, not equal copies
+            for lst in (gw.emb, gw.proj, gw.ln_gamma, gw.ln_beta, gw.head):
+                lst[l] = lst[1]
+    else:
+        sw, ow, gw = _setup(cfg)
     ctx, tok = synth.make_draft_inputs(cfg)
     h = B.spec_create(gw)
     B.spec_set_option(h, B.SPEC_OPT_GEMM_IMPL, impl)
@@ -156,7 +168,9 @@ def _draft_and_check(B, cfg, seqs=None, impl=0, check_levels=False):
         for l in range(cfg.n if chk.tolerated == 0 else 1):
             S = ws_view(ws, lay.state[l], N * cfg.d_inner, torch.bfloat16).view(N, cfg.d_inner)
             S = S.to(torch.float32).cpu().numpy()
-            assert np.allclose(S, dd.states[l], rtol=0.008, atol=2e-4), f"level {l} states"
+            # not teacher-forced: a one-ulp bf16 difference at one level perturbs the next level's input,
+            # so the allowance grows with the depth (the per-level check in DraftChecker is the strict one)
+            assert np.allclose(S, dd.states[l], rtol=0.008 * (1 + l), atol=2e-4 * (1 + l)), f"level {l} states"
             N *= cfg.topk[l]
             if chk.tolerated == 0:
                 t = ws_view(ws, lay.tok[l + 1], N, torch.int32).cpu().numpy()
@@ -180,6 +194,29 @@ def test_draft_odd_shapes(B, topk, K, Bn, V, d_base, d):
     cfg = small_cfg(d_base=d_base, d_inner=d, V=V, topk=topk, K=K, B=Bn, seed=len(topk) + Bn)
     chk = _draft_and_check(B, cfg, check_levels=True)
     assert chk.tolerated <= max(1, Bn // 5)
+
+
+@pytest.mark.parametrize("topk,K", [((3, 2, 2, 1, 1), 9), ((2, 2, 2, 1, 1, 1, 1), 8), ((2, 1, 2, 1, 2, 1, 2, 1), 16)])
+def test_draft_code_model_head_counts(B, topk, K):
+    """5, 7 (the code models of Sec. 4.3 / 4.4) and the maximum of 8 heads."""
+    cfg = small_cfg(d_base=96, d_inner=128, V=3000, topk=topk, K=K, B=3, seed=40 + len(topk))
+    chk = _draft_and_check(B, cfg, check_levels=True)
+    assert chk.tolerated <= 1
+
+
+def test_draft_weight_tied_heads(B):
+    cfg = small_cfg(d_base=128, d_inner=128, V=2048, topk=(3, 2, 2, 2), K=10, B=4, seed=77)
+    chk = _draft_and_check(B, cfg, check_levels=True, tie_weights=True)
+    assert chk.tolerated <= 1
+
+
+def test_draft_single_candidate_at_production_width(B):
+    """k = 1 (Sec. 4.2 / Sec. 5: the setting the paper recommends under load): topk = 1 at every head,
+    one candidate per sequence, at the Llama2-7B-shaped widths."""
+    import dataclasses
+    cfg = dataclasses.replace(synth.CONFIGS["llama2-7b"], topk=(1, 1, 1), K=1, B=4)
+    chk = _draft_and_check(B, cfg)
+    assert chk.tolerated <= 1
 
 
 def test_draft_llama2_7b_shape(B):
