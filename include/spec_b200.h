@@ -50,9 +50,11 @@ enum spec_option {
                                   kernels kept for debugging the tensor-core path              */
     SPEC_OPT_HEAD_BLOCK_N = 1, /* vocabulary columns per tile of the head GEMM; 0 = automatic  */
     SPEC_OPT_PROJ_BLOCK_N = 2, /* output columns per tile of the state projection; 0 = auto    */
-    SPEC_OPT_PROFILE = 3       /* 1: spec_draft brackets each of its kernels with CUDA events on
+    SPEC_OPT_PROFILE = 3,      /* 1: spec_draft brackets each of its kernels with CUDA events on
                                   the caller's stream (read them with spec_profile_read); costs a
                                   few microseconds per call, off by default                    */
+    SPEC_OPT_FP8_MAX_ROWS = 4  /* levels with at most this many nodes use the e4m3 copy of their head when
+                                  one is attached (default 128; 0 = never)                     */
 };
 
 typedef struct spec_handle_s *spec_handle_t;
@@ -81,6 +83,7 @@ typedef struct {
     uint64_t score[SPEC_MAX_HEADS + 1];   /* fp32  [N_l]: cumulative log-prob, level l>=1     */
     uint64_t state[SPEC_MAX_HEADS];       /* bf16  [N_l, d_inner]: post-GELU state of level l */
     uint64_t proj;                        /* fp32  [max rows, d_inner]: projected parent states */
+    uint64_t state8, state8_scale;        /* e4m3 [rows, d_inner] + fp32 [rows]: states of an e4m3 level */
     uint64_t part_val, part_idx, part_ms; /* per-tile partial top-k lists and (max, sum-exp)  */
     uint64_t logits;                      /* fp32 [max N_l, V]; only with SPEC_OPT_GEMM_IMPL=1 */
     int32_t block_n[SPEC_MAX_HEADS];      /* vocabulary columns per head-GEMM tile            */
@@ -174,6 +177,23 @@ int spec_verify_early(const int32_t *cand_tok, const void *base_logits, int logi
 #define SPEC_VERIFY_STATIC_SCRATCH_BYTES (1u << 20)
 int spec_verify_static(const int32_t *cand_tok, const void *base_logits, int logits_dtype, int B, int K, int n,
                        int V, int32_t *accept_len, int32_t *best_cand, int32_t *next_tok, void *cuda_stream);
+
+/* ---- e4m3 copy of a vocabulary head (optional) ---------------------------------------------
+ * (The paper runs everything in 16 bits; this is an implementation option for the heads whose
+ * cost is reading the weights: levels with few nodes.)  A head's bf16 matrix [V, d_inner] can be
+ * given a second form, e4m3 bytes [V, d_inner] with one fp32 scale per vocabulary row, half the
+ * bytes.  For a level that has it and at most SPEC_OPT_FP8_MAX_ROWS nodes, spec_draft multiplies
+ * in e4m3 (tensor cores, fp32 accumulation), keeps the 16 tokens with the best APPROXIMATE logits
+ * per node, recomputes those 16 logits exactly from the bf16 weights and states, and branches
+ * to the top-k of the exact values; only the softmax normaliser comes from the approximate
+ * logits (its error is of order 1e-3 in log-probability).  d_inner must be a multiple of 16.
+ *   spec_quantize_head  fills q_out (dev, V * d_inner bytes, 16-byte aligned) and scale_out
+ *                       (dev fp32 [V]) from head `level`'s bf16 weights on `cuda_stream`
+ *   spec_set_head_fp8   attaches such a pair to the handle (caller-owned, must outlive the calls
+ *                       that use it); q = NULL detaches
+ */
+int spec_quantize_head(spec_handle_t h, int level, void *q_out, float *scale_out, void *cuda_stream);
+int spec_set_head_fp8(spec_handle_t h, int level, const void *q, const float *scale);
 
 /* Per-kernel device times of the last spec_draft issued with SPEC_OPT_PROFILE = 1, in launch
  * order: for every head (projection GEMM, mix/LayerNorm/GELU, head GEMM, merge/expand), then

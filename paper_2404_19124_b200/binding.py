@@ -20,13 +20,13 @@ MAX_HEADS, MAX_TOPK, MAX_LEAVES = 8, 8, 4096
  SPEC_ERR_TIMEOUT, SPEC_ERR_NO_DEVICE, SPEC_ERR_STATIC_SCRATCH) = range(9)
 SPEC_VERIFY_STATIC_SCRATCH_BYTES = 1 << 20
 SPEC_BF16, SPEC_F32 = 0, 1
-SPEC_OPT_GEMM_IMPL, SPEC_OPT_HEAD_BLOCK_N, SPEC_OPT_PROJ_BLOCK_N, SPEC_OPT_PROFILE = 0, 1, 2, 3
+SPEC_OPT_GEMM_IMPL, SPEC_OPT_HEAD_BLOCK_N, SPEC_OPT_PROJ_BLOCK_N, SPEC_OPT_PROFILE, SPEC_OPT_FP8_MAX_ROWS = 0, 1, 2, 3, 4
 
 EXPORTS = [
     "spec_version", "spec_status_str", "spec_last_cuda_error", "spec_create", "spec_destroy", "spec_set_option",
     "spec_draft_workspace_bytes", "spec_draft_layout", "spec_draft", "spec_verify_workspace_bytes", "spec_verify",
     "spec_profile_read", "spec_poll_error", "spec_head_workspace_bytes", "spec_head_logits", "spec_head_topk",
-    "spec_verify_static", "spec_verify_early",
+    "spec_verify_static", "spec_verify_early", "spec_quantize_head", "spec_set_head_fp8",
 ]
 
 if not os.path.exists(LIB_PATH):
@@ -51,7 +51,7 @@ class SpecDraftLayoutC(C.Structure):
     _fields_ = [
         ("total_bytes", C.c_uint64), ("error_word", C.c_uint64),
         ("tok", C.c_uint64 * (MAX_HEADS + 1)), ("score", C.c_uint64 * (MAX_HEADS + 1)),
-        ("state", C.c_uint64 * MAX_HEADS), ("proj", C.c_uint64),
+        ("state", C.c_uint64 * MAX_HEADS), ("proj", C.c_uint64), ("state8", C.c_uint64), ("state8_scale", C.c_uint64),
         ("part_val", C.c_uint64), ("part_idx", C.c_uint64), ("part_ms", C.c_uint64), ("logits", C.c_uint64),
         ("block_n", C.c_int32 * MAX_HEADS), ("n_tiles", C.c_int32 * MAX_HEADS),
     ]
@@ -76,6 +76,8 @@ _lib.spec_verify.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_int, 
 _lib.spec_verify_static.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_int, C.c_int, C.c_int,
                                     C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
 _lib.spec_verify_early.argtypes = _lib.spec_verify.argtypes
+_lib.spec_quantize_head.argtypes = [C.c_void_p, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p]
+_lib.spec_set_head_fp8.argtypes = [C.c_void_p, C.c_int, C.c_void_p, C.c_void_p]
 _lib.spec_poll_error.argtypes = [C.c_void_p, C.c_void_p]
 _lib.spec_profile_read.argtypes = [C.c_void_p, C.POINTER(C.c_float), C.c_int, C.POINTER(C.c_int)]
 _lib.spec_head_workspace_bytes.restype = C.c_size_t
@@ -281,6 +283,27 @@ def spec_verify_static(cand_tok: torch.Tensor, base_logits: torch.Tensor, accept
     with torch.cuda.device(cand_tok.device):
         _check(_lib.spec_verify_static(_ptr(cand_tok), _ptr(base_logits), dt, B, K, n, V, _ptr(accept_len),
                                        _ptr(best_cand), _ptr(next_tok), _stream_ptr(stream)), "spec_verify_static")
+
+
+def spec_attach_fp8_heads(h: SpecHandle, levels: Optional[Sequence[int]] = None,
+                          stream: Optional[torch.cuda.Stream] = None) -> None:
+    """Quantises the heads of `levels` (default: all) to e4m3 (spec_quantize_head) into tensors the handle
+    keeps alive and attaches them (spec_set_head_fp8).  Allocation happens here, in the caller's framework,
+    not in the library."""
+    if not hasattr(h, "_fp8"):
+        h._fp8 = {}
+    for l in (range(h.n_heads) if levels is None else levels):
+        q = torch.empty((h.V, h.d_inner), dtype=torch.uint8, device=h.device)
+        sc = torch.empty(h.V, dtype=torch.float32, device=h.device)
+        _check(_lib.spec_quantize_head(h.ptr, int(l), _ptr(q), _ptr(sc), _stream_ptr(stream)), "spec_quantize_head")
+        _check(_lib.spec_set_head_fp8(h.ptr, int(l), _ptr(q), _ptr(sc)), "spec_set_head_fp8")
+        h._fp8[int(l)] = (q, sc)
+
+
+def spec_detach_fp8_heads(h: SpecHandle) -> None:
+    for l in range(h.n_heads):
+        _check(_lib.spec_set_head_fp8(h.ptr, int(l), None, None), "spec_set_head_fp8")
+    h._fp8 = {}
 
 
 def spec_profile_read(h: SpecHandle) -> List[float]:

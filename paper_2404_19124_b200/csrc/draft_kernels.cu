@@ -94,14 +94,8 @@ prune_kernel(const float *leaf_score, PruneArgs pa, int L, int Lpad, int K, int3
 
 }  // namespace
 
-int launch_mix_ln_gelu(const float *P, int p_splits, size_t p_split_stride, const void *emb, const int32_t *tok,
-                       const float *gamma, const float *beta, int rows, int d_inner, int V, int parent_div, float a,
-                       float b, float eps, void *S_out, int32_t *err, cudaStream_t st) {
-    MixArgs m{};
-    m.P = P; m.p_splits = p_splits; m.p_split_stride = p_split_stride;
-    m.emb = (const uint16_t *)emb; m.tok = tok; m.gamma = gamma; m.beta = beta;
-    m.d = d_inner; m.V = V; m.parent_div = parent_div; m.a = a; m.b = b; m.eps = eps;
-    m.S_out = (uint16_t *)S_out; m.err = err;
+int launch_mix_ln_gelu(const MixArgs &m, int rows, cudaStream_t st) {
+    const int d_inner = m.d;
     if (d_inner <= 8 * kRowThreads * 2 && rows > num_sms()) {
         SPEC_CUDA_TRY(launch_pdl(mix_ln_gelu_many_kernel, dim3(rows), dim3(kRowThreads), 0, st, m));
     } else if (d_inner <= 8 * kRowThreads * 2) {

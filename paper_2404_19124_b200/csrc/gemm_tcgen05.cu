@@ -92,14 +92,16 @@ EncodeTiledFn get_encode_fn() {
 
 }  // namespace
 
-int make_tmap(CUtensorMap *map, const void *base, uint64_t rows, uint64_t cols, uint32_t box_rows, bool streamed) {
+int make_tmap(CUtensorMap *map, const void *base, uint64_t rows, uint64_t cols, uint32_t box_rows, bool streamed,
+              bool fp8) {
     EncodeTiledFn fn = get_encode_fn();
     if (!fn) return SPEC_ERR_CUDA;
+    const uint32_t esz = fp8 ? 1 : 2;
     cuuint64_t dims[2] = {cols, rows};
-    cuuint64_t strides[1] = {cols * 2};
-    cuuint32_t box[2] = {(cuuint32_t)kBlockK, box_rows};
+    cuuint64_t strides[1] = {cols * esz};
+    cuuint32_t box[2] = {(cuuint32_t)(kSlabBytes / esz), box_rows};
     cuuint32_t estr[2] = {1, 1};
-    CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(base), dims, strides, box, estr,
+    CUresult r = fn(map, fp8 ? CU_TENSOR_MAP_DATA_TYPE_UINT8 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(base), dims, strides, box, estr,
                     CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
                     streamed ? CU_TENSOR_MAP_L2_PROMOTION_L2_256B : CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
@@ -133,13 +135,16 @@ int choose_block_n(int M, int N, int num_sm, bool prefer_wide) {
 }
 
 int plan_job(tc::GemmJob *j, int M, int N, int Kd, int block_n, const GemmEpilogue &epi) {
-    if (M <= 0 || N <= 0 || Kd <= 0 || Kd % 8 != 0 || block_n < 32 || block_n > 256 || block_n % 32 != 0)
-        return SPEC_ERR_SHAPE;
+    const int fp8 = epi.fp8 ? 1 : 0;
+    if (M <= 0 || N <= 0 || Kd <= 0 || Kd % (fp8 ? 16 : 8) != 0 || block_n < 32 || block_n > 256 || block_n % 32 != 0)
+        return SPEC_ERR_SHAPE;   // rows are whole 16-byte units
     j->M = M; j->N = N; j->Kd = Kd;
     j->block_n = block_n;
     j->m_tiles = (M + kBlockM - 1) / kBlockM;
     j->n_tiles = (N + block_n - 1) / block_n;
-    const int num_kb = (Kd + kBlockK - 1) / kBlockK;
+    j->fp8 = fp8;
+    const int ke = fp8 ? kSlabBytes : kSlabBytes / 2;
+    const int num_kb = (Kd + ke - 1) / ke;
     j->splits = epi.mode == 2 && epi.splits > 1 ? epi.splits : 1;
     j->kb_per_split = (num_kb + j->splits - 1) / j->splits;
     if ((j->splits - 1) * j->kb_per_split >= num_kb) return SPEC_ERR_SHAPE;   // every split must own a K block
@@ -163,9 +168,10 @@ int launch_gemm_tc_jobs(const GemmCall *calls, int n_calls, int32_t *err, cudaSt
         int rc = plan_job(&p.job[q], c.M, c.N, c.Kd, c.block_n, c.epi);
         if (rc != SPEC_OK) return rc;
         if (((uintptr_t)c.A & 15) || ((uintptr_t)c.B & 15)) return SPEC_ERR_INVALID_ARG;
-        rc = make_tmap(&maps.a[q], c.A, (uint64_t)c.M, (uint64_t)c.Kd, kBlockM, p.job[q].w_is_a != 0);
+        rc = make_tmap(&maps.a[q], c.A, (uint64_t)c.M, (uint64_t)c.Kd, kBlockM, p.job[q].w_is_a != 0, p.job[q].fp8 != 0);
         if (rc != SPEC_OK) return rc;
-        rc = make_tmap(&maps.b[q], c.B, (uint64_t)c.N, (uint64_t)c.Kd, (uint32_t)c.block_n, p.job[q].w_is_a == 0);
+        rc = make_tmap(&maps.b[q], c.B, (uint64_t)c.N, (uint64_t)c.Kd, (uint32_t)c.block_n, p.job[q].w_is_a == 0,
+                       p.job[q].fp8 != 0);
         if (rc != SPEC_OK) return rc;
         if (c.block_n > max_block_n) max_block_n = c.block_n;
         total_tiles += (long long)p.job[q].m_tiles * p.job[q].n_tiles * p.job[q].splits;
@@ -176,7 +182,7 @@ int launch_gemm_tc_jobs(const GemmCall *calls, int n_calls, int32_t *err, cudaSt
         p.job[q].first_cta = (int)(offset % grid);
         offset += (long long)p.job[q].m_tiles * p.job[q].n_tiles * p.job[q].splits;
     }
-    p.slot_bytes = (uint32_t)kABytes + (uint32_t)max_block_n * kBlockK * 2;
+    p.slot_bytes = (uint32_t)kABytes + (uint32_t)max_block_n * kSlabBytes;
     const int budget = kSmemLimit - 1024 - (int)sizeof(Barriers) - 64;
     p.stages = budget / (int)p.slot_bytes;
     if (p.stages > kMaxStages) p.stages = kMaxStages;

@@ -13,21 +13,30 @@
 
 #include <math.h>
 
+#include "fp8.cuh"
 #include "spec_common.cuh"
 
 namespace spec {
 namespace rows {
+
+using spec::MergeArgs;
+using spec::MixArgs;
 
 struct BlockSync {
     static __device__ __forceinline__ void sync() { __syncthreads(); }
 };
 
 // Scratch in shared memory for one group.
+constexpr int kMaxGroupWarps = 16;
+constexpr int kMaxRounds = 16;        // most entries a selection can return (top-k itself needs at most 8)
 struct Scratch {
     float red[32];
-    float red_m[8], red_s[8];
-    uint32_t cand_k[2][8];
-    int cand_i[2][8];
+    float red_m[kMaxGroupWarps], red_s[kMaxGroupWarps];
+    uint32_t cand_k[2][kMaxGroupWarps];
+    int cand_i[2][kMaxGroupWarps];
+    float out_val[kMaxRounds];        // result of merge_select: values, best first ...
+    int out_id[kMaxRounds];           // ... and their token ids
+    float lse;
 };
 
 template <int kThreads, typename Sync>
@@ -44,22 +53,23 @@ __device__ __forceinline__ float group_sum(float v, float *red, int tid) {
     return t;
 }
 
+template <int kThreads, typename Sync>
+__device__ __forceinline__ float group_max(float v, float *red, int tid) {
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, off));
+    const int w = tid >> 5, l = tid & 31;
+    Sync::sync();
+    if (l == 0) red[w] = v;
+    Sync::sync();
+    float t = (l < kThreads / 32) ? red[l] : 0.0f;   // used for magnitudes only
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) t = fmaxf(t, __shfl_xor_sync(0xffffffffu, t, off));
+    return t;
+}
+
 // Exact (erf) GELU.  erff is kept out of line: inlined it would be the bulk of the row step's code.
 static __device__ __noinline__ float erf_call(float x) { return erff(x); }
 __device__ __forceinline__ float gelu_erf(float y) { return 0.5f * y * (1.0f + erf_call(y * 0.70710678118654752440f)); }
-
-struct MixArgs {
-    const float *P;            // `p_splits` partial projections, `p_split_stride` floats apart: [parent rows, d] each
-    int p_splits;
-    size_t p_split_stride;
-    const uint16_t *emb;       // bf16 [V, d]
-    const int32_t *tok;        // [rows]
-    const float *gamma, *beta; // fp32 [d]
-    int d, V, parent_div;
-    float a, b, eps;
-    uint16_t *S_out;           // bf16 [rows, d]
-    int32_t *err;
-};
 
 // Node r of the level.  Siblings share a projected parent state: parent(r) = r / parent_div.
 // h = a * P[parent] + b * E[tok[r]].  The row lives in registers: thread t owns the 8-element groups
@@ -156,6 +166,7 @@ __device__ __forceinline__ void mix_ln_gelu_row(const MixArgs &m, int r, int tid
     }
     const float var = group_sum<kThreads, Sync>(sq, red, tid) / (float)d;
     const float rstd = rsqrtf(var + m.eps);
+    float amax = 0.0f;   // largest magnitude of the bf16-rounded state (for the e4m3 copy); h is reused for it
 #pragma unroll
     for (int it = 0; it < kIters; ++it) {
         const int i = (it * kThreads + tid) * 8;
@@ -175,8 +186,21 @@ __device__ __forceinline__ void mix_ln_gelu_row(const MixArgs &m, int r, int tid
             const float s0 = gelu_erf((h[it][j] - mean) * rstd * gv[j] + bv[j]);
             const float s1 = gelu_erf((h[it][j + 1] - mean) * rstd * gv[j + 1] + bv[j + 1]);
             packed[j >> 1] = float_to_bf16_bits(s0) | (float_to_bf16_bits(s1) << 16);
+            h[it][j] = i < d ? __uint_as_float(packed[j >> 1] << 16) : 0.0f;
+            h[it][j + 1] = i < d ? __uint_as_float(packed[j >> 1] & 0xffff0000u) : 0.0f;
+            amax = fmaxf(amax, fmaxf(fabsf(h[it][j]), fabsf(h[it][j + 1])));
         }
         if (i < d) *(uint4 *)(m.S_out + (size_t)r * d + i) = make_uint4(packed[0], packed[1], packed[2], packed[3]);
+    }
+    if (m.S8_out != nullptr) {   // uniform over the group
+        const float scale = row_scale_of(group_max<kThreads, Sync>(amax, red, tid));
+        const float inv = 1.0f / scale;
+#pragma unroll
+        for (int it = 0; it < kIters; ++it) {
+            const int i = (it * kThreads + tid) * 8;
+            if (i < d) *(uint2 *)(m.S8_out + (size_t)r * d + i) = e4m3x8(h[it], inv);
+        }
+        if (tid == 0) m.s8_scale[r] = scale;
     }
 }
 
@@ -211,16 +235,6 @@ __device__ __forceinline__ uint32_t float_key(float v) {
 __device__ __forceinline__ float key_float(uint32_t k) {
     return __uint_as_float((k & 0x80000000u) ? (k & 0x7fffffffu) : ~k);
 }
-
-struct MergeArgs {
-    const float *part_val;     // [rows, n_tiles, SPEC_MAX_TOPK] (first `topk` of each list valid, any order)
-    const int32_t *part_idx;   // same shape
-    const float *part_ms;      // [rows, n_tiles, 2] = (max, sum of exp(x - max))
-    int n_tiles, topk;
-    const float *score_in;     // [rows] or null (score 0)
-    int32_t *tok_out;          // [rows, topk]
-    float *score_out;          // [rows, topk]
-};
 
 // Sorts one tile's list (8 slots, any order, slots >= topk ignored) best first with a fixed network and
 // folds it into the sorted list (tv, ti): with both lists sorted, "the better of a[i] and b[7 - i]" keeps
@@ -273,19 +287,21 @@ __device__ __forceinline__ void fold_max_sum(float &m, float &s, const float2 &m
 }
 
 // Thread t folds the lists of tiles t, t + kThreads, ... into one sorted list of 8 in registers, two
-// tiles per trip with all ten loads issued before the first is used.  The group then extracts the `topk`
-// best in `topk` rounds; a round is two warp-wide integer reductions (redux.sync: maximum of the value
-// keys, then minimum token id among the lanes that hold it) and one shared-memory exchange between warps.
+// tiles per trip with all ten loads issued before the first is used.  The group then extracts the
+// `rounds` best (rounds <= kMaxRounds) in as many rounds; a round is two warp-wide integer reductions
+// (redux.sync: maximum of the value keys, then minimum token id among the lanes that hold it) and one
+// shared-memory exchange between the warps.  Results: sc->out_val / out_id (best first; exhausted slots
+// hold -inf / 0x7fffffff) and sc->lse, valid for the whole group after the function returns.
 template <int kThreads, typename Sync>
-__device__ __forceinline__ void merge_expand_row(const MergeArgs &g, int r, int tid, Scratch *sc) {
+__device__ __forceinline__ void merge_select(const MergeArgs &g, int r, int tid, Scratch *sc, int rounds) {
     constexpr int kWarps = kThreads / 32;
     constexpr int kT = SPEC_MAX_TOPK;
+    static_assert(kWarps <= kMaxGroupWarps, "scratch arrays");
     const int lane = tid & 31, warp = tid >> 5;
-    const int n_tiles = g.n_tiles, topk = g.topk;
-    const float4 *pv4 = (const float4 *)(g.part_val + (size_t)r * g.n_tiles * kT);
-    const int4 *pi4 = (const int4 *)(g.part_idx + (size_t)r * g.n_tiles * kT);
-    const float2 *pms = (const float2 *)(g.part_ms + (size_t)r * g.n_tiles * 2);
-    const float base = (g.score_in) ? __ldcg(g.score_in + r) : 0.0f;
+    const int n_tiles = g.n_tiles, topk = g.list_len > 0 ? g.list_len : g.topk;   // slots to read per list
+    const float4 *pv4 = (const float4 *)(g.part_val + (size_t)r * n_tiles * kT);
+    const int4 *pi4 = (const int4 *)(g.part_idx + (size_t)r * n_tiles * kT);
+    const float2 *pms = (const float2 *)(g.part_ms + (size_t)r * n_tiles * 2);
 
     float tv[kT];
     int ti[kT];
@@ -316,7 +332,7 @@ __device__ __forceinline__ void merge_expand_row(const MergeArgs &g, int r, int 
     float ws = (m > -INFINITY) ? s * __expf(m - wm) : 0.0f;
 #pragma unroll
     for (int off = 16; off > 0; off >>= 1) ws += __shfl_xor_sync(0xffffffffu, ws, off);
-    Sync::sync();   // the scratch may still be read by a previous call's last round
+    Sync::sync();   // the scratch may still be read by a previous call
     if (lane == 0) {
         sc->red_m[warp] = wm;
         sc->red_s[warp] = ws;
@@ -329,9 +345,9 @@ __device__ __forceinline__ void merge_expand_row(const MergeArgs &g, int r, int 
 #pragma unroll
     for (int w = 0; w < kWarps; ++w)
         if (sc->red_m[w] > -INFINITY) bs += sc->red_s[w] * __expf(sc->red_m[w] - bm);
-    const float lse = bm + logf(bs);
+    if (tid == 0) sc->lse = bm + logf(bs);
 
-    for (int j = 0; j < topk; ++j) {
+    for (int j = 0; j < rounds; ++j) {
         const uint32_t my_key = float_key(tv[0]);
         const uint32_t wk = __reduce_max_sync(0xffffffffu, my_key);
         const uint32_t wi = __reduce_min_sync(0xffffffffu, my_key == wk ? (uint32_t)ti[0] : 0xffffffffu);
@@ -361,9 +377,21 @@ __device__ __forceinline__ void merge_expand_row(const MergeArgs &g, int r, int 
             ti[kT - 1] = 0x7fffffff;
         }
         if (tid == 0) {
-            g.tok_out[(size_t)r * topk + j] = bi;
-            g.score_out[(size_t)r * topk + j] = base + (key_float(bk) - lse);
+            sc->out_val[j] = key_float(bk);
+            sc->out_id[j] = bi;
         }
+    }
+    Sync::sync();
+}
+
+// The row's top-k tokens and log-probabilities become its children.
+template <int kThreads, typename Sync>
+__device__ __forceinline__ void merge_expand_row(const MergeArgs &g, int r, int tid, Scratch *sc) {
+    const float base = (tid < g.topk && g.score_in) ? __ldcg(g.score_in + r) : 0.0f;   // in flight during the merge
+    merge_select<kThreads, Sync>(g, r, tid, sc, g.topk);
+    if (tid < g.topk) {
+        g.tok_out[(size_t)r * g.topk + tid] = sc->out_id[tid];
+        g.score_out[(size_t)r * g.topk + tid] = base + (sc->out_val[tid] - sc->lse);
     }
 }
 

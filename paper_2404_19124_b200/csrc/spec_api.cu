@@ -35,6 +35,9 @@ struct spec_handle_s {
     int head_block_n;
     int proj_block_n;
     int profile;
+    int fp8_max_rows;                      // SPEC_OPT_FP8_MAX_ROWS
+    const void *head8[SPEC_MAX_HEADS];     // e4m3 copies of the heads (caller-owned), null: none
+    const float *head8_scale[SPEC_MAX_HEADS];
     int prof_count;                        // events recorded by the last profiled draft
     cudaEvent_t prof_ev[kMaxProfEvents];   // created when profiling is switched on
 };
@@ -53,6 +56,7 @@ struct DraftPlan {
     spec_draft_layout_t lay;
     int proj_block_n[SPEC_MAX_HEADS];
     int proj_splits[SPEC_MAX_HEADS];   // > 0: swapped split-K projection (few parent rows); 0: plain
+    bool use_fp8[SPEC_MAX_HEADS];      // the level's head runs on the e4m3 copy of its weights
 };
 
 int head_block_n_for(const spec_handle_s *h, int rows) {
@@ -126,6 +130,15 @@ int make_draft_plan(const spec_handle_s *h, int B, const int32_t *topk, int K, D
     }
     y.proj = off;
     off = align_up(off + sizeof(float) * max_proj_floats, kWsAlign);
+    int max_fp8_rows = 0;
+    for (int l = 0; l < p->n; ++l) {
+        p->use_fp8[l] = h->gemm_impl == 0 && !h->profile && h->head8[l] != nullptr && p->N[l] <= h->fp8_max_rows;
+        if (p->use_fp8[l] && p->N[l] > max_fp8_rows) max_fp8_rows = p->N[l];
+    }
+    y.state8 = off;
+    off = align_up(off + (size_t)max_fp8_rows * w.d_inner, kWsAlign);
+    y.state8_scale = off;
+    off = align_up(off + sizeof(float) * (size_t)max_fp8_rows, kWsAlign);
     y.part_val = off;
     off = align_up(off + sizeof(float) * max_part_units * SPEC_MAX_TOPK, kWsAlign);
     y.part_idx = off;
@@ -220,6 +233,11 @@ int spec_create(spec_handle_t *out, const spec_weights_t *w) {
     h->head_block_n = 0;
     h->proj_block_n = 0;
     h->profile = 0;
+    h->fp8_max_rows = 128;
+    for (int l = 0; l < SPEC_MAX_HEADS; ++l) {
+        h->head8[l] = nullptr;
+        h->head8_scale[l] = nullptr;
+    }
     h->prof_count = 0;
     for (cudaEvent_t &e : h->prof_ev) e = nullptr;
     *out = h;
@@ -254,9 +272,30 @@ int spec_set_option(spec_handle_t h, int option, int value) {
             h->profile = value;
             h->prof_count = 0;
             return SPEC_OK;
+        case SPEC_OPT_FP8_MAX_ROWS:
+            if (value < 0 || value > 128) return SPEC_ERR_INVALID_ARG;
+            h->fp8_max_rows = value;
+            return SPEC_OK;
         default:
             return SPEC_ERR_INVALID_ARG;
     }
+}
+
+int spec_quantize_head(spec_handle_t h, int level, void *q_out, float *scale_out, void *cuda_stream) {
+    if (!h || !q_out || !scale_out) return SPEC_ERR_INVALID_ARG;
+    if (level < 0 || level >= h->w.n_heads || h->w.d_inner % 16 != 0) return SPEC_ERR_SHAPE;
+    if ((uintptr_t)q_out & 15) return SPEC_ERR_INVALID_ARG;
+    return launch_quantize_rows(h->w.head[level], h->w.V, h->w.d_inner, q_out, scale_out, (cudaStream_t)cuda_stream);
+}
+
+int spec_set_head_fp8(spec_handle_t h, int level, const void *q, const float *scale) {
+    if (!h) return SPEC_ERR_INVALID_ARG;
+    if (level < 0 || level >= h->w.n_heads) return SPEC_ERR_SHAPE;
+    if (q != nullptr && (scale == nullptr || ((uintptr_t)q & 15) || ((uintptr_t)scale & 15) || h->w.d_inner % 16 != 0))
+        return SPEC_ERR_INVALID_ARG;
+    h->head8[level] = q;
+    h->head8_scale[level] = q ? scale : nullptr;
+    return SPEC_OK;
 }
 
 int spec_profile_read(spec_handle_t h, float *ms_out, int max_count, int *count_out) {
@@ -363,9 +402,18 @@ int spec_draft(spec_handle_t h, const void *ctx_state, const int32_t *last_tok, 
         }
         SPEC_PROF_MARK();
         // gather + mix + LayerNorm + GELU -> bf16 state of every node of this level
-        rc = launch_mix_ln_gelu(P, splits > 0 ? splits : 1, split_stride, w.emb[l], tok_l, w.ln_gamma[l],
-                                w.ln_beta[l], rows, w.d_inner, w.V, l == 0 ? 1 : topk[l - 1], w.state_weight,
-                                w.emb_weight, w.ln_eps, S, err, st);
+        const bool fp8 = p.use_fp8[l];
+        MixArgs mx{};
+        mx.P = P; mx.p_splits = splits > 0 ? splits : 1; mx.p_split_stride = split_stride;
+        mx.emb = (const uint16_t *)w.emb[l]; mx.tok = tok_l; mx.gamma = w.ln_gamma[l]; mx.beta = w.ln_beta[l];
+        mx.d = w.d_inner; mx.V = w.V; mx.parent_div = l == 0 ? 1 : topk[l - 1];
+        mx.a = w.state_weight; mx.b = w.emb_weight; mx.eps = w.ln_eps;
+        mx.S_out = (uint16_t *)S; mx.err = err;
+        if (fp8) {   // the head of this level reads the states as e4m3
+            mx.S8_out = (uint8_t *)(ws + p.lay.state8);
+            mx.s8_scale = (float *)(ws + p.lay.state8_scale);
+        }
+        rc = launch_mix_ln_gelu(mx, rows, st);
         if (rc != SPEC_OK) return rc;
         SPEC_PROF_MARK();
         // vocabulary head with the fused per-tile top-k / log-sum-exp epilogue.  The next level's
@@ -373,7 +421,7 @@ int spec_draft(spec_handle_t h, const void *ctx_state, const int32_t *last_tok, 
         // launch: its weight tiles follow the head's through the same ring and one kernel boundary less
         // lies on the critical path (with per-kernel profiling it stays a launch of its own).
         proj_done = false;
-        if (h->gemm_impl == 0 && !h->profile && l + 1 < p.n) {
+        if (h->gemm_impl == 0 && !h->profile && (l + 1 < p.n || fp8)) {
             GemmCall c[2];
             c[0].A = S; c[0].B = w.head[l]; c[0].M = rows; c[0].N = w.V; c[0].Kd = w.d_inner;
             c[0].block_n = p.lay.block_n[l];
@@ -381,9 +429,18 @@ int spec_draft(spec_handle_t h, const void *ctx_state, const int32_t *last_tok, 
             c[0].epi.mode = 1;
             c[0].epi.part_val = part_val; c[0].epi.part_idx = part_idx; c[0].epi.part_ms = part_ms;
             c[0].epi.topk = topk[l];
-            c[1] = proj_call(l + 1);
-            rc = launch_gemm_tc_jobs(c, 2, err, st);
-            proj_done = true;
+            if (fp8) {   // e4m3 operands; every tile keeps SPEC_MAX_TOPK candidates by approximate logit
+                c[0].A = ws + p.lay.state8;
+                c[0].B = h->head8[l];
+                c[0].epi.fp8 = 1;
+                c[0].epi.topk = SPEC_MAX_TOPK;
+                c[0].epi.row_scale = (const float *)(ws + p.lay.state8_scale);
+                c[0].epi.col_scale = h->head8_scale[l];
+            }
+            const bool pair = l + 1 < p.n;
+            if (pair) c[1] = proj_call(l + 1);
+            rc = launch_gemm_tc_jobs(c, pair ? 2 : 1, err, st);
+            proj_done = pair;
         } else {
             rc = run_head_partials(h, S, w.head[l], rows, p.lay.block_n[l], topk[l], part_val, part_idx, part_ms,
                                    logits_scratch, err, st);
@@ -391,11 +448,23 @@ int spec_draft(spec_handle_t h, const void *ctx_state, const int32_t *last_tok, 
         if (rc != SPEC_OK) return rc;
         SPEC_PROF_MARK();
         // fold the partials, branch: children (token, cumulative score) of every node
-        rc = launch_merge_expand(part_val, part_idx, part_ms, rows, p.lay.n_tiles[l], topk[l], score_l,
-                                 (int32_t *)(ws + p.lay.tok[l + 1]), (float *)(ws + p.lay.score[l + 1]), st);
+        if (fp8) {
+            // short list by approximate logit, exact re-scoring from the bf16 weights, then the children
+            MergeArgs g{};
+            g.part_val = part_val; g.part_idx = part_idx; g.part_ms = part_ms;
+            g.n_tiles = p.lay.n_tiles[l]; g.topk = topk[l]; g.list_len = SPEC_MAX_TOPK;
+            g.score_in = score_l;
+            g.tok_out = (int32_t *)(ws + p.lay.tok[l + 1]);
+            g.score_out = (float *)(ws + p.lay.score[l + 1]);
+            rc = launch_merge_rescore(g, w.head[l], S, rows, w.d_inner, w.V, st);
+        } else {
+            rc = launch_merge_expand(part_val, part_idx, part_ms, rows, p.lay.n_tiles[l], topk[l], score_l,
+                                     (int32_t *)(ws + p.lay.tok[l + 1]), (float *)(ws + p.lay.score[l + 1]), st);
+        }
         if (rc != SPEC_OK) return rc;
         SPEC_PROF_MARK();
     }
+
     PruneArgs pa{};
     pa.n = p.n;
     for (int l = 0; l < p.n; ++l) {

@@ -102,6 +102,9 @@ struct GemmEpilogue {
     int32_t *part_idx; // mode 1: [M, n_tiles, SPEC_MAX_TOPK]
     float *part_ms;    // mode 1: [M, n_tiles, 2]
     int topk;          // mode 1
+    int fp8;           // operands are e4m3 bytes instead of bf16; mode 1 then multiplies every accumulator by
+                       // row_scale[m] * col_scale[n] before the selection
+    const float *row_scale, *col_scale;
 };
 int choose_block_n(int M, int N, int num_sm, bool tensor_bound_pref);
 int launch_gemm_tc(const void *A, const void *B, int M, int N, int Kd, int block_n, const GemmEpilogue &epi,
@@ -120,11 +123,39 @@ int launch_gemm_simt(const void *A, const void *B, int M, int N, int Kd, float *
 int launch_partials_from_logits(const float *logits, int M, int N, int block_n, int topk, float *part_val,
                                 int32_t *part_idx, float *part_ms, cudaStream_t st);
 
-// ---- row kernels of the draft (draft_kernels.cu) ----------------------------------------
-// P: `p_splits` partial projections, `p_split_stride` floats apart, summed on load.
-int launch_mix_ln_gelu(const float *P, int p_splits, size_t p_split_stride, const void *emb, const int32_t *tok,
-                       const float *gamma, const float *beta, int rows, int d_inner, int V, int parent_div, float a,
-                       float b, float eps, void *S_out, int32_t *err, cudaStream_t st);
+// ---- row-wise steps of the draft (row_ops.cuh, draft_kernels.cu, fp8_kernels.cu) ---------
+struct MixArgs {
+    const float *P;            // `p_splits` partial projections, `p_split_stride` floats apart: [parent rows, d] each
+    int p_splits;
+    size_t p_split_stride;
+    const uint16_t *emb;       // bf16 [V, d]
+    const int32_t *tok;        // [rows]
+    const float *gamma, *beta; // fp32 [d]
+    int d, V, parent_div;
+    float a, b, eps;
+    uint16_t *S_out;           // bf16 [rows, d]
+    uint8_t *S8_out;           // optional: the same states as e4m3 bytes [rows, d] ...
+    float *s8_scale;           // ... with one scale per row [rows] (see fp8.cuh); null: not written
+    int32_t *err;
+};
+
+struct MergeArgs {
+    const float *part_val;     // [rows, n_tiles, SPEC_MAX_TOPK] (first `topk` of each list valid, any order)
+    const int32_t *part_idx;   // same shape
+    const float *part_ms;      // [rows, n_tiles, 2] = (max, sum of exp(x - max))
+    int n_tiles, topk;
+    int list_len;              // valid slots of every partial list; 0: the same as topk
+    const float *score_in;     // [rows] or null (score 0)
+    int32_t *tok_out;          // [rows, topk]
+    float *score_out;          // [rows, topk]
+};
+
+// e4m3 copy of a bf16 matrix: Q [rows, d] bytes and one fp32 scale per row (fp8.cuh).
+int launch_quantize_rows(const void *X, int rows, int d, void *Q, float *scale, cudaStream_t st);
+// merge of approximate partial lists + exact re-scoring of the short list + expansion (fp8_kernels.cu)
+int launch_merge_rescore(const MergeArgs &g, const void *W, const void *S, int rows, int d, int V, cudaStream_t st);
+
+int launch_mix_ln_gelu(const MixArgs &m, int rows, cudaStream_t st);
 int launch_merge_expand(const float *part_val, const int32_t *part_idx, const float *part_ms, int rows, int n_tiles,
                         int topk, const float *score_in, int32_t *tok_out, float *score_out, cudaStream_t st);
 struct PruneArgs {

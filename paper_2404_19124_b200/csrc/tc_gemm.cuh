@@ -23,12 +23,12 @@ namespace spec {
 namespace tc {
 
 constexpr int kBlockM = 128;
-constexpr int kBlockK = 64;            // 64 bf16 = 128 bytes = one swizzle span
-constexpr int kUmmaK = 16;
+constexpr int kSlabBytes = 128;        // one K block = one 128-byte swizzle span per row: 64 bf16 or 128 fp8 elements
+constexpr int kUmmaBytes = 32;         // K extent of one MMA instruction in bytes: 16 bf16 or 32 fp8 elements
 constexpr int kThreads = 192;
 constexpr int kEpilogueThreads = 128;  // warps 2-5
 constexpr int kMaxStages = 12;
-constexpr int kABytes = kBlockM * kBlockK * 2;
+constexpr int kABytes = kBlockM * kSlabBytes;
 constexpr int kSmemLimit = 222 * 1024; // leaves room on the SM for the small kernels that overlap with a GEMM
 constexpr uint32_t kSpinFast = 1u << 14;
 constexpr uint32_t kSpinMax = 1u << 24;
@@ -47,6 +47,7 @@ struct GemmJob {
     int M, N, Kd;
     int block_n, m_tiles, n_tiles;
     int splits, kb_per_split;   // split-K: tile = (m_tile, n_tile, split), split slowest
+    int fp8;                    // 0: bf16 operands (kind::f16); 1: e4m3 operands (kind::f8f6f4); fp32 accumulation either way
     int w_is_a;                 // 1: A holds the weights (no kernel writes them), B the states; 0: the reverse
     int first_cta;              // CTA that takes tile 0; tile t goes to CTA (first_cta + t) mod grid
     GemmEpilogue epi;
@@ -125,12 +126,13 @@ __device__ __forceinline__ uint64_t make_smem_desc(uint32_t saddr) {
     return d;
 }
 
-// Instruction descriptor for kind::f16: D = fp32, A = B = bf16, both K-major, M x N tile.
-__device__ __forceinline__ uint32_t make_instr_desc(int m, int n) {
+// Instruction descriptor: D = fp32, A and B of one type (bf16 for kind::f16, e4m3 for kind::f8f6f4), both
+// K-major, M x N tile.
+__device__ __forceinline__ uint32_t make_instr_desc(int m, int n, bool fp8) {
     uint32_t d = 0;
     d |= 1u << 4;                      // D format: F32
-    d |= 1u << 7;                      // A format: BF16
-    d |= 1u << 10;                     // B format: BF16
+    d |= (fp8 ? 0u : 1u) << 7;         // A format: kind::f16: 1 = BF16; kind::f8f6f4: 0 = E4M3
+    d |= (fp8 ? 0u : 1u) << 10;        // B format, same encoding
     d |= (uint32_t)(n >> 3) << 17;     // N / 8
     d |= (uint32_t)(m >> 4) << 24;     // M / 16
     return d;
@@ -142,6 +144,16 @@ __device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t adesc, uint6
         "{\n\t.reg .pred p;\n\t"
         "setp.ne.b32 p, %4, 0;\n\t"
         "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+
+__device__ __forceinline__ void umma_e4m3(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
+                                          uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f8f6f4 [%0], %1, %2, %3, p;\n\t}"
         ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
         : "memory");
 }
@@ -228,6 +240,10 @@ __device__ __forceinline__ void pipe_teardown(const Pipe &pp, int tmem_cols) {
     }
 }
 
+// Elements of one 128-byte K block, and the number of K blocks of a job.
+__device__ __forceinline__ int slab_elems(const GemmJob &j) { return j.fp8 ? kSlabBytes : kSlabBytes / 2; }
+__device__ __forceinline__ int num_k_blocks(const GemmJob &j) { return (j.Kd + slab_elems(j) - 1) / slab_elems(j); }
+
 __device__ __forceinline__ int first_tile_of(const GemmJob &j) {
     return (int)((blockIdx.x + gridDim.x - (unsigned)j.first_cta % gridDim.x) % gridDim.x);
 }
@@ -245,10 +261,10 @@ __device__ __forceinline__ void advance(const Pipe &pp, RingPos &rp) {
 template <typename DepWait>
 __device__ __forceinline__ bool produce_job(const Pipe &pp, const GemmJob &j, const CUtensorMap *tmap_a,
                                             const CUtensorMap *tmap_b, RingPos &rp, int &issued, DepWait dep_wait) {
-    const int num_kb = (j.Kd + kBlockK - 1) / kBlockK;
+    const int num_kb = num_k_blocks(j), ke = slab_elems(j);
     const int mn_tiles = j.m_tiles * j.n_tiles;
     const int num_tiles = mn_tiles * j.splits;
-    const uint32_t tx = (uint32_t)kABytes + (uint32_t)j.block_n * kBlockK * 2;
+    const uint32_t tx = (uint32_t)kABytes + (uint32_t)j.block_n * kSlabBytes;
     const int first = first_tile_of(j);
     if (first >= num_tiles) return true;
     Barriers *bars = pp.bars;
@@ -263,8 +279,8 @@ __device__ __forceinline__ bool produce_job(const Pipe &pp, const GemmJob &j, co
             if (!mbar_wait(&bars->empty[q.stage], q.phase ^ 1u, bars, pp.err)) return false;
             uint8_t *sa = pp.tiles + (size_t)q.stage * pp.slot_bytes;
             mbar_arrive_expect_tx(&bars->full[q.stage], tx);
-            if (j.w_is_a) tma_load_2d(sa, tmap_a, (kb0 + i) * kBlockK, m_tile * kBlockM, &bars->full[q.stage]);
-            else tma_load_2d(sa + kABytes, tmap_b, (kb0 + i) * kBlockK, n_tile * j.block_n, &bars->full[q.stage]);
+            if (j.w_is_a) tma_load_2d(sa, tmap_a, (kb0 + i) * ke, m_tile * kBlockM, &bars->full[q.stage]);
+            else tma_load_2d(sa + kABytes, tmap_b, (kb0 + i) * ke, n_tile * j.block_n, &bars->full[q.stage]);
             advance(pp, q);
         }
     }
@@ -282,8 +298,8 @@ __device__ __forceinline__ bool produce_job(const Pipe &pp, const GemmJob &j, co
                 if (!mbar_wait(&bars->empty[rp.stage], rp.phase ^ 1u, bars, pp.err)) return false;
                 mbar_arrive_expect_tx(&bars->full[rp.stage], tx);
             }
-            if (!prefetched || !j.w_is_a) tma_load_2d(sa, tmap_a, kb * kBlockK, m_tile * kBlockM, &bars->full[rp.stage]);
-            if (!prefetched || j.w_is_a) tma_load_2d(sb, tmap_b, kb * kBlockK, n_tile * j.block_n, &bars->full[rp.stage]);
+            if (!prefetched || !j.w_is_a) tma_load_2d(sa, tmap_a, kb * ke, m_tile * kBlockM, &bars->full[rp.stage]);
+            if (!prefetched || j.w_is_a) tma_load_2d(sb, tmap_b, kb * ke, n_tile * j.block_n, &bars->full[rp.stage]);
             ++done;
             ++issued;
             advance(pp, rp);
@@ -303,10 +319,10 @@ __device__ __forceinline__ void producer_drain(const Pipe &pp, RingPos rp, int i
 
 // ---- MMA issuer (one thread) ----------------------------------------------------------------------
 __device__ __forceinline__ bool mma_job(const Pipe &pp, const GemmJob &j, RingPos &rp, AccPos &ap) {
-    const int num_kb = (j.Kd + kBlockK - 1) / kBlockK;
+    const int num_kb = num_k_blocks(j);
     const int mn_tiles = j.m_tiles * j.n_tiles;
     const int num_tiles = mn_tiles * j.splits;
-    const uint32_t idesc = make_instr_desc(kBlockM, j.block_n);
+    const uint32_t idesc = make_instr_desc(kBlockM, j.block_n, j.fp8 != 0);
     Barriers *bars = pp.bars;
     for (int tile = first_tile_of(j); tile < num_tiles; tile += gridDim.x) {
         if (!mbar_wait(&bars->acc_empty[ap.acc], ap.phase ^ 1u, bars, pp.err)) return false;
@@ -320,10 +336,12 @@ __device__ __forceinline__ bool mma_job(const Pipe &pp, const GemmJob &j, RingPo
             const uint32_t sa = smem_u32(pp.tiles + (size_t)rp.stage * pp.slot_bytes);
             const uint32_t sb = sa + kABytes;
 #pragma unroll
-            for (int k = 0; k < kBlockK / kUmmaK; ++k) {
-                const uint64_t adesc = make_smem_desc(sa + k * kUmmaK * 2);
-                const uint64_t bdesc = make_smem_desc(sb + k * kUmmaK * 2);
-                umma_bf16(tmem_d, adesc, bdesc, idesc, ((kb - kb0) | k) != 0 ? 1u : 0u);
+            for (int k = 0; k < kSlabBytes / kUmmaBytes; ++k) {
+                const uint64_t adesc = make_smem_desc(sa + k * kUmmaBytes);
+                const uint64_t bdesc = make_smem_desc(sb + k * kUmmaBytes);
+                const uint32_t acc = ((kb - kb0) | k) != 0 ? 1u : 0u;
+                if (j.fp8) umma_e4m3(tmem_d, adesc, bdesc, idesc, acc);
+                else umma_bf16(tmem_d, adesc, bdesc, idesc, acc);
             }
             umma_commit(&bars->empty[rp.stage]);   // frees the slot once these MMAs have read it
             advance(pp, rp);
@@ -341,6 +359,21 @@ __device__ __forceinline__ bool mma_job(const Pipe &pp, const GemmJob &j, RingPo
 //           kept sorted by a min/max network (new_v[j] = max(v[j], min(v[j-1], x)));
 //   pass 2  re-reads the tile from TMEM and emits the columns whose value reaches the topk-th
 //           largest; equal values are taken in ascending column order, exactly `topk` entries.
+// e4m3 operands: accumulator -> logit, v[i] * row_scale * col_scale[col0 + c + i] (columns past N untouched).
+__device__ __forceinline__ void scale_chunk(float (&v)[32], float rs, const float *cs, int valid) {
+    if (valid >= 32 && (((uintptr_t)cs) & 15) == 0) {
+#pragma unroll
+        for (int i = 0; i < 32; i += 4) {
+            const float4 q = *(const float4 *)(cs + i);
+            v[i] *= rs * q.x; v[i + 1] *= rs * q.y; v[i + 2] *= rs * q.z; v[i + 3] *= rs * q.w;
+        }
+    } else {
+#pragma unroll
+        for (int i = 0; i < 32; ++i)
+            if (i < valid) v[i] *= rs * cs[i];
+    }
+}
+
 template <int kCap>
 __device__ __forceinline__ void epilogue_topk(const GemmJob &p, uint32_t taddr, int row, bool row_ok, int col0,
                                               int n_tile) {
@@ -349,10 +382,12 @@ __device__ __forceinline__ void epilogue_topk(const GemmJob &p, uint32_t taddr, 
 #pragma unroll
     for (int j = 0; j < kCap; ++j) best[j] = -INFINITY;
     float run_m = -INFINITY, run_s = 0.0f;
+    const float rs = (p.fp8 && row_ok) ? p.epi.row_scale[row] : 1.0f;
     for (int c = 0; c < p.block_n; c += 32) {
         float v[32];
         tmem_ld32(taddr + c, v);
         const int valid = p.N - (col0 + c);   // columns of this chunk inside the vocabulary
+        if (p.fp8) scale_chunk(v, rs, p.epi.col_scale + col0 + c, valid);
         if (valid < 32) {
 #pragma unroll
             for (int i = 0; i < 32; ++i)
@@ -406,6 +441,7 @@ __device__ __forceinline__ void epilogue_topk(const GemmJob &p, uint32_t taddr, 
         float v[32];
         tmem_ld32(taddr + c, v);
         const int valid = p.N - (col0 + c);
+        if (p.fp8) scale_chunk(v, rs, p.epi.col_scale + col0 + c, valid);
         // candidates of this chunk as a bit mask: no per-element branches
         uint32_t mask = 0;
 #pragma unroll
@@ -511,9 +547,10 @@ __device__ __forceinline__ bool epilogue_job(const Pipe &pp, const GemmJob &j, A
 }  // namespace tc
 
 // ---- host side (gemm_tcgen05.cu) ---------------------------------------------------------------
-// 2-D bf16 row-major [rows, cols] tensor, box = [box_rows, 64 columns], 128-byte swizzle; `streamed`
-// marks the operand that is read once from HBM (wider L2 fetches).
-int make_tmap(CUtensorMap *map, const void *base, uint64_t rows, uint64_t cols, uint32_t box_rows, bool streamed);
+// 2-D row-major [rows, cols] tensor of bf16 (or, `fp8`, of bytes), box = [box_rows, 128 bytes], 128-byte
+// swizzle; `streamed` marks the operand that is read once from HBM (wider L2 fetches).
+int make_tmap(CUtensorMap *map, const void *base, uint64_t rows, uint64_t cols, uint32_t box_rows, bool streamed,
+              bool fp8 = false);
 // Fills the tiling fields of a job (m_tiles, n_tiles, splits, kb_per_split, w_is_a) from its shape and epilogue.
 int plan_job(tc::GemmJob *j, int M, int N, int Kd, int block_n, const GemmEpilogue &epi);
 

@@ -118,7 +118,7 @@ def test_head_topk_exact_ties_prefer_lower_token_id(B):
     B.spec_destroy(h)
 
 
-def _draft_and_check(B, cfg, seqs=None, impl=0, check_levels=False, tie_weights=False):
+def _draft_and_check(B, cfg, seqs=None, impl=0, check_levels=False, tie_weights=False, fp8=False):
     """Runs spec_draft at the config's full batch and compares the sequences in `seqs`
     (default: all) with the oracle, one sequence at a time (sequences are independent).
     tie_weights: every head after the first aliases the second head's tensors (the weight-tied
@@ -137,6 +137,8 @@ def _draft_and_check(B, cfg, seqs=None, impl=0, check_levels=False, tie_weights=
     ctx, tok = synth.make_draft_inputs(cfg)
     h = B.spec_create(gw)
     B.spec_set_option(h, B.SPEC_OPT_GEMM_IMPL, impl)
+    if fp8:      # levels of up to 128 nodes multiply in e4m3 and re-score a short list exactly
+        B.spec_attach_fp8_heads(h)
     cand_tok, cand_logp, ws = B.spec_draft(h, ctx.cuda(), tok.cuda(), cfg.topk, cfg.K)
     assert B.spec_poll_error(ws) == 0
     ct, lp = cand_tok.cpu().numpy(), cand_logp.cpu().numpy()
@@ -217,6 +219,54 @@ def test_draft_single_candidate_at_production_width(B):
     cfg = dataclasses.replace(synth.CONFIGS["llama2-7b"], topk=(1, 1, 1), K=1, B=4)
     chk = _draft_and_check(B, cfg)
     assert chk.tolerated <= 1
+
+
+def test_quantize_head_is_rowwise_e4m3(B):
+    """spec_quantize_head against the format's definition written with library casts: one scale per
+    vocabulary row, max|row| / 448, and round-to-nearest-even e4m3 of row / scale."""
+    cfg = small_cfg(d_base=64, d_inner=160, V=777, topk=(2, 2), seed=5)
+    sw, ow, gw = _setup(cfg)
+    gw.head[1][5].zero_()                                # an all-zero row keeps scale 1
+    h = B.spec_create(gw)
+    B.spec_attach_fp8_heads(h, levels=[1])
+    q, sc = h._fp8[1]
+    w = gw.head[1].to(torch.float32)
+    amax = w.abs().amax(dim=1)
+    want_sc = torch.where(amax > 0, torch.div(amax, torch.full_like(amax, 448.0)), torch.ones_like(amax))   # true division
+    assert torch.equal(sc, want_sc)
+    want_q = (w * torch.div(torch.ones_like(want_sc), want_sc)[:, None]).to(torch.float8_e4m3fn).view(torch.uint8)
+    assert torch.equal(q, want_q)
+    B.spec_destroy(h)
+
+
+@pytest.mark.parametrize("topk,K,Bn,V,d_base,d", [((4, 3, 2), 8, 1, 1024, 256, 256), ((3, 2, 2), 5, 7, 1000, 80, 64),
+                                                   ((8, 8), 64, 2, 2048, 128, 192), ((6, 4, 3), 32, 4, 8000, 96, 512)])
+def test_draft_fp8_heads_small_shapes(B, topk, K, Bn, V, d_base, d):
+    """e4m3 head + exact re-scoring of the short list: same protocol and tolerances as the bf16 path."""
+    cfg = small_cfg(d_base=d_base, d_inner=d, V=V, topk=topk, K=K, B=Bn, seed=3 * len(topk) + Bn)
+    # the normaliser comes from approximate logits (error ~1e-3), so leaves with nearly equal scores may
+    # swap places against the oracle; every such list goes through the level-by-level check in DraftChecker
+    chk = _draft_and_check(B, cfg, check_levels=False, fp8=True)
+    assert chk.exact + chk.tolerated == Bn
+
+
+@pytest.mark.parametrize("name,seqs", [("llama2-7b", (0, 3, 7)), ("llama2-13b", (1, 9))])
+def test_draft_fp8_heads_full_size(B, name, seqs):
+    """Full batch at the benchmark shapes with the e4m3 heads on the weight-bound levels; the oracle
+    re-computes whole trees for a sample of sequences, and the candidates agree with the bf16 path's."""
+    cfg = synth.CONFIGS[name]
+    _draft_and_check(B, cfg, seqs=seqs, fp8=True)
+    sw, ow, gw = _setup(cfg)
+    ctx, tok = synth.make_draft_inputs(cfg)
+    h = B.spec_create(gw)
+    ref_tok, ref_lp, _ = B.spec_draft(h, ctx.cuda(), tok.cuda(), cfg.topk, cfg.K)
+    B.spec_attach_fp8_heads(h)
+    got_tok, got_lp, ws = B.spec_draft(h, ctx.cuda(), tok.cuda(), cfg.topk, cfg.K)
+    assert B.spec_poll_error(ws) == 0
+    same = (ref_tok == got_tok).all(dim=2).all(dim=1)
+    assert same.float().mean().item() >= 0.75, "most sequences must give identical candidate lists"
+    assert (ref_lp[same] - got_lp[same]).abs().max().item() <= cfg.n * 5e-3
+    B.spec_destroy(h)
 
 
 def test_draft_llama2_7b_shape(B):
