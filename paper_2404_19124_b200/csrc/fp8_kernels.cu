@@ -5,7 +5,7 @@
 //   head GEMM           kind::f8f6f4 on the two e4m3 operands; the epilogue rescales the accumulators
 //                       and keeps, per vocabulary tile, 8 candidates by APPROXIMATE logit and the
 //                       (max, sum-exp) of the approximate logits
-//   merge_rescore       folds the tiles' lists into a short list of kShortList tokens per row and the
+//   merge_rescore       folds the tiles' lists into a short list of 8 to 16 tokens per row and the
 //                       row's log-sum-exp, recomputes the short-listed logits EXACTLY from the bf16
 //                       weights and states (fp32 accumulation, as the bf16 head does), and takes the
 //                       top-k of those
@@ -71,20 +71,35 @@ __global__ void __launch_bounds__(kRescoreThreads) merge_rescore_kernel(RescoreA
     griddep_wait();
     const int r = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const float base = (tid == 0 && a.merge.score_in) ? __ldcg(a.merge.score_in + r) : 0.0f;
-    merge_select<kRescoreThreads, BlockSync>(a.merge, r, tid, &sc, kShortList);
+    // short list: twice the branching factor plus two, at least 8, at most one per warp
+    const int n_short = min(kShortList, max(8, 2 * a.merge.topk + 2));
+    merge_select<kRescoreThreads, BlockSync>(a.merge, r, tid, &sc, n_short);
     // exact logit of short-listed token `warp`: dot product of two bf16 rows, fp32 accumulation
-    const int v = sc.out_id[warp];
+    const int v = warp < n_short ? sc.out_id[warp] : -1;
     float acc = 0.0f;
     if (v >= 0 && v < a.V) {
         const uint16_t *w = a.W + (size_t)v * a.d, *s = a.S + (size_t)r * a.d;
-        for (int i = lane * 8; i < a.d; i += 32 * 8) {
-            const uint4 qw = *(const uint4 *)(w + i);
-            const uint4 qs = __ldcg((const uint4 *)(s + i));
-            const uint32_t ww[4] = {qw.x, qw.y, qw.z, qw.w}, ss[4] = {qs.x, qs.y, qs.z, qs.w};
+        constexpr int kBatch = 8;   // 8-element groups per lane whose loads are in flight together
+        for (int i0 = lane * 8; i0 < a.d; i0 += 32 * 8 * kBatch) {
+            uint4 qw[kBatch], qs[kBatch];
 #pragma unroll
-            for (int j = 0; j < 4; ++j) {
-                acc = fmaf(__uint_as_float(ww[j] << 16), __uint_as_float(ss[j] << 16), acc);
-                acc = fmaf(__uint_as_float(ww[j] & 0xffff0000u), __uint_as_float(ss[j] & 0xffff0000u), acc);
+            for (int u = 0; u < kBatch; ++u) {
+                const int i = i0 + u * 32 * 8;
+                qw[u] = make_uint4(0u, 0u, 0u, 0u);
+                qs[u] = qw[u];
+                if (i < a.d) {
+                    qw[u] = *(const uint4 *)(w + i);
+                    qs[u] = __ldcg((const uint4 *)(s + i));
+                }
+            }
+#pragma unroll
+            for (int u = 0; u < kBatch; ++u) {
+                const uint32_t ww[4] = {qw[u].x, qw[u].y, qw[u].z, qw[u].w}, ss[4] = {qs[u].x, qs[u].y, qs[u].z, qs[u].w};
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    acc = fmaf(__uint_as_float(ww[j] << 16), __uint_as_float(ss[j] << 16), acc);
+                    acc = fmaf(__uint_as_float(ww[j] & 0xffff0000u), __uint_as_float(ss[j] & 0xffff0000u), acc);
+                }
             }
         }
     }
@@ -94,8 +109,8 @@ __global__ void __launch_bounds__(kRescoreThreads) merge_rescore_kernel(RescoreA
     __syncthreads();
     // warp 0: the top-k of the exact logits, (value desc, token id asc)
     if (warp == 0) {
-        float val = lane < kShortList ? exact[lane] : -INFINITY;
-        int id = lane < kShortList ? sc.out_id[lane] : 0x7fffffff;
+        float val = lane < n_short ? exact[lane] : -INFINITY;
+        int id = lane < n_short ? sc.out_id[lane] : 0x7fffffff;
         const float lse = sc.lse;
         const int topk = a.merge.topk;
         for (int j = 0; j < topk; ++j) {

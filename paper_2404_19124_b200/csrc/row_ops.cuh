@@ -338,14 +338,17 @@ __device__ __forceinline__ void merge_select(const MergeArgs &g, int r, int tid,
         sc->red_s[warp] = ws;
     }
     Sync::sync();
-    float bm = sc->red_m[0];
+    if (warp == 0) {   // one lane per warp's (max, sum): a second shuffle reduction
+        const float pm = lane < kWarps ? sc->red_m[lane] : -INFINITY;
+        const float ps = lane < kWarps ? sc->red_s[lane] : 0.0f;
+        float bm = pm;
 #pragma unroll
-    for (int w = 1; w < kWarps; ++w) bm = fmaxf(bm, sc->red_m[w]);
-    float bs = 0.0f;
+        for (int off = 16; off > 0; off >>= 1) bm = fmaxf(bm, __shfl_xor_sync(0xffffffffu, bm, off));
+        float bs = pm > -INFINITY ? ps * __expf(pm - bm) : 0.0f;
 #pragma unroll
-    for (int w = 0; w < kWarps; ++w)
-        if (sc->red_m[w] > -INFINITY) bs += sc->red_s[w] * __expf(sc->red_m[w] - bm);
-    if (tid == 0) sc->lse = bm + logf(bs);
+        for (int off = 16; off > 0; off >>= 1) bs += __shfl_xor_sync(0xffffffffu, bs, off);
+        if (lane == 0) sc->lse = bm + logf(bs);
+    }
 
     for (int j = 0; j < rounds; ++j) {
         const uint32_t my_key = float_key(tv[0]);
@@ -356,17 +359,11 @@ __device__ __forceinline__ void merge_select(const MergeArgs &g, int r, int tid,
             sc->cand_i[j & 1][warp] = (int)wi;
         }
         Sync::sync();   // rounds alternate between two buffers, so one barrier per round is enough
-        uint32_t bk = sc->cand_k[j & 1][0];
-        int bi = sc->cand_i[j & 1][0];
-#pragma unroll
-        for (int w = 1; w < kWarps; ++w) {
-            const uint32_t ok = sc->cand_k[j & 1][w];
-            const int oi = sc->cand_i[j & 1][w];
-            if (ok > bk || (ok == bk && oi < bi)) {
-                bk = ok;
-                bi = oi;
-            }
-        }
+        // every warp reduces the warps' candidates again, one per lane: two more redux instead of a scan
+        const uint32_t ck = lane < kWarps ? sc->cand_k[j & 1][lane] : 0u;
+        const uint32_t ci = lane < kWarps ? (uint32_t)sc->cand_i[j & 1][lane] : 0xffffffffu;
+        const uint32_t bk = __reduce_max_sync(0xffffffffu, ck);
+        const int bi = (int)__reduce_min_sync(0xffffffffu, (lane < kWarps && ck == bk) ? ci : 0xffffffffu);
         if (ti[0] == bi && my_key == bk) {   // token ids are unique, so exactly one thread owns a real entry
 #pragma unroll
             for (int q = 0; q < kT - 1; ++q) {

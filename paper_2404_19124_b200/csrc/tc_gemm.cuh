@@ -138,26 +138,6 @@ __device__ __forceinline__ uint32_t make_instr_desc(int m, int n, bool fp8) {
     return d;
 }
 
-__device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
-                                          uint32_t accumulate) {
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "setp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-        ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
-        : "memory");
-}
-
-__device__ __forceinline__ void umma_e4m3(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
-                                          uint32_t accumulate) {
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "setp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::f8f6f4 [%0], %1, %2, %3, p;\n\t}"
-        ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
-        : "memory");
-}
-
 __device__ __forceinline__ void umma_commit(uint64_t *bar) {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar))
                  : "memory");
@@ -318,11 +298,56 @@ __device__ __forceinline__ void producer_drain(const Pipe &pp, RingPos rp, int i
 }
 
 // ---- MMA issuer (one thread) ----------------------------------------------------------------------
-__device__ __forceinline__ bool mma_job(const Pipe &pp, const GemmJob &j, RingPos &rp, AccPos &ap) {
+// The four MMAs of one K block in one instruction sequence.  The single issuing thread is on the
+// critical path of the tensor pipe, so the loop around this does as little as possible: descriptors are
+// (constant high word, start address >> 4 in the low word), and consecutive MMAs advance the low words by
+// 32 bytes >> 4 = 2.  `first_acc` = 0 makes the first MMA overwrite the accumulator (start of a tile).
+template <bool kFp8>
+__device__ __forceinline__ void umma_k_block(uint32_t tmem_d, uint32_t lo_a, uint32_t lo_b, uint32_t desc_hi,
+                                             uint32_t idesc, uint32_t first_acc) {
+#define SPEC_MMA_SEQ(KIND)                                                                  \
+    asm volatile(                                                                           \
+        "{\n\t"                                                                             \
+        ".reg .pred p, t;\n\t"                                                              \
+        ".reg .b64 da, db;\n\t"                                                             \
+        ".reg .b32 la, lb;\n\t"                                                             \
+        "setp.ne.b32 p, %5, 0;\n\t"                                                         \
+        "setp.eq.b32 t, 0, 0;\n\t"                                                          \
+        "mov.b64 da, {%1, %3};\n\t"                                                         \
+        "mov.b64 db, {%2, %3};\n\t"                                                         \
+        "tcgen05.mma.cta_group::1.kind::" KIND " [%0], da, db, %4, p;\n\t"                  \
+        "add.u32 la, %1, 2;\n\t"                                                            \
+        "add.u32 lb, %2, 2;\n\t"                                                            \
+        "mov.b64 da, {la, %3};\n\t"                                                         \
+        "mov.b64 db, {lb, %3};\n\t"                                                         \
+        "tcgen05.mma.cta_group::1.kind::" KIND " [%0], da, db, %4, t;\n\t"                  \
+        "add.u32 la, %1, 4;\n\t"                                                            \
+        "add.u32 lb, %2, 4;\n\t"                                                            \
+        "mov.b64 da, {la, %3};\n\t"                                                         \
+        "mov.b64 db, {lb, %3};\n\t"                                                         \
+        "tcgen05.mma.cta_group::1.kind::" KIND " [%0], da, db, %4, t;\n\t"                  \
+        "add.u32 la, %1, 6;\n\t"                                                            \
+        "add.u32 lb, %2, 6;\n\t"                                                            \
+        "mov.b64 da, {la, %3};\n\t"                                                         \
+        "mov.b64 db, {lb, %3};\n\t"                                                         \
+        "tcgen05.mma.cta_group::1.kind::" KIND " [%0], da, db, %4, t;\n\t"                  \
+        "}"                                                                                 \
+        ::"r"(tmem_d), "r"(lo_a), "r"(lo_b), "r"(desc_hi), "r"(idesc), "r"(first_acc)      \
+        : "memory")
+    if (kFp8) SPEC_MMA_SEQ("f8f6f4");
+    else SPEC_MMA_SEQ("f16");
+#undef SPEC_MMA_SEQ
+}
+
+template <bool kFp8>
+__device__ __forceinline__ bool mma_job_kind(const Pipe &pp, const GemmJob &j, RingPos &rp, AccPos &ap) {
+    static_assert(kSlabBytes / kUmmaBytes == 4, "umma_k_block issues four MMAs");
     const int num_kb = num_k_blocks(j);
     const int mn_tiles = j.m_tiles * j.n_tiles;
     const int num_tiles = mn_tiles * j.splits;
-    const uint32_t idesc = make_instr_desc(kBlockM, j.block_n, j.fp8 != 0);
+    const uint32_t idesc = make_instr_desc(kBlockM, j.block_n, kFp8);
+    const uint32_t desc_hi = (uint32_t)(make_smem_desc(0) >> 32);
+    const uint32_t lo_base = (smem_u32(pp.tiles) & 0x3ffffu) >> 4, lo_slot = pp.slot_bytes >> 4;
     Barriers *bars = pp.bars;
     for (int tile = first_tile_of(j); tile < num_tiles; tile += gridDim.x) {
         if (!mbar_wait(&bars->acc_empty[ap.acc], ap.phase ^ 1u, bars, pp.err)) return false;
@@ -330,19 +355,13 @@ __device__ __forceinline__ bool mma_job(const Pipe &pp, const GemmJob &j, RingPo
         const uint32_t tmem_d = pp.tmem_base + (uint32_t)(ap.acc * pp.acc_stride);
         const int split = tile / mn_tiles;
         const int kb0 = split * j.kb_per_split, kb1 = min(num_kb, kb0 + j.kb_per_split);
+        uint32_t acc = 0u;
         for (int kb = kb0; kb < kb1; ++kb) {
             if (!mbar_wait(&bars->full[rp.stage], rp.phase, bars, pp.err)) return false;
             tc_fence_after();
-            const uint32_t sa = smem_u32(pp.tiles + (size_t)rp.stage * pp.slot_bytes);
-            const uint32_t sb = sa + kABytes;
-#pragma unroll
-            for (int k = 0; k < kSlabBytes / kUmmaBytes; ++k) {
-                const uint64_t adesc = make_smem_desc(sa + k * kUmmaBytes);
-                const uint64_t bdesc = make_smem_desc(sb + k * kUmmaBytes);
-                const uint32_t acc = ((kb - kb0) | k) != 0 ? 1u : 0u;
-                if (j.fp8) umma_e4m3(tmem_d, adesc, bdesc, idesc, acc);
-                else umma_bf16(tmem_d, adesc, bdesc, idesc, acc);
-            }
+            const uint32_t lo_a = lo_base + (uint32_t)rp.stage * lo_slot;
+            umma_k_block<kFp8>(tmem_d, lo_a, lo_a + (kABytes >> 4), desc_hi, idesc, acc);
+            acc = 1u;
             umma_commit(&bars->empty[rp.stage]);   // frees the slot once these MMAs have read it
             advance(pp, rp);
         }
@@ -350,6 +369,10 @@ __device__ __forceinline__ bool mma_job(const Pipe &pp, const GemmJob &j, RingPo
         if (++ap.acc == 2) { ap.acc = 0; ap.phase ^= 1u; }
     }
     return true;
+}
+
+__device__ __forceinline__ bool mma_job(const Pipe &pp, const GemmJob &j, RingPos &rp, AccPos &ap) {
+    return j.fp8 ? mma_job_kind<true>(pp, j, rp, ap) : mma_job_kind<false>(pp, j, rp, ap);
 }
 
 // ---- epilogue, mode 1 -----------------------------------------------------------------------------
@@ -374,7 +397,7 @@ __device__ __forceinline__ void scale_chunk(float (&v)[32], float rs, const floa
     }
 }
 
-template <int kCap>
+template <int kCap, bool kFp8>
 __device__ __forceinline__ void epilogue_topk(const GemmJob &p, uint32_t taddr, int row, bool row_ok, int col0,
                                               int n_tile) {
     constexpr float kLog2e = 1.4426950408889634f;
@@ -382,12 +405,12 @@ __device__ __forceinline__ void epilogue_topk(const GemmJob &p, uint32_t taddr, 
 #pragma unroll
     for (int j = 0; j < kCap; ++j) best[j] = -INFINITY;
     float run_m = -INFINITY, run_s = 0.0f;
-    const float rs = (p.fp8 && row_ok) ? p.epi.row_scale[row] : 1.0f;
+    const float rs = (kFp8 && row_ok) ? p.epi.row_scale[row] : 1.0f;
     for (int c = 0; c < p.block_n; c += 32) {
         float v[32];
         tmem_ld32(taddr + c, v);
         const int valid = p.N - (col0 + c);   // columns of this chunk inside the vocabulary
-        if (p.fp8) scale_chunk(v, rs, p.epi.col_scale + col0 + c, valid);
+        if (kFp8) scale_chunk(v, rs, p.epi.col_scale + col0 + c, valid);
         if (valid < 32) {
 #pragma unroll
             for (int i = 0; i < 32; ++i)
@@ -441,7 +464,7 @@ __device__ __forceinline__ void epilogue_topk(const GemmJob &p, uint32_t taddr, 
         float v[32];
         tmem_ld32(taddr + c, v);
         const int valid = p.N - (col0 + c);
-        if (p.fp8) scale_chunk(v, rs, p.epi.col_scale + col0 + c, valid);
+        if (kFp8) scale_chunk(v, rs, p.epi.col_scale + col0 + c, valid);
         // candidates of this chunk as a bit mask: no per-element branches
         uint32_t mask = 0;
 #pragma unroll
@@ -533,8 +556,9 @@ __device__ __forceinline__ bool epilogue_job(const Pipe &pp, const GemmJob &j, A
                 }
             }
         } else {
-            if (j.epi.topk <= 4) epilogue_topk<4>(j, taddr, row, row_ok, col0, n_tile);
-            else epilogue_topk<SPEC_MAX_TOPK>(j, taddr, row, row_ok, col0, n_tile);
+            if (j.fp8) epilogue_topk<SPEC_MAX_TOPK, true>(j, taddr, row, row_ok, col0, n_tile);
+            else if (j.epi.topk <= 4) epilogue_topk<4, false>(j, taddr, row, row_ok, col0, n_tile);
+            else epilogue_topk<SPEC_MAX_TOPK, false>(j, taddr, row, row_ok, col0, n_tile);
         }
         tc_fence_before();
         __syncwarp();
