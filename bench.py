@@ -376,6 +376,26 @@ def main():
     torch.cuda.synchronize()
     bk_ms = v0.elapsed_time(v1) / prof_steps
 
+    # the same step with e4m3 copies of the heads attached (used by the levels of up to 128 nodes)
+    B.spec_attach_fp8_heads(h)
+    ws8 = torch.empty(B.spec_draft_workspace_bytes(h, Bn, cfg.topk, K), dtype=torch.uint8, device=dev)
+
+    def step8(i):
+        B.spec_draft(h, ctx, tok, cfg.topk, K, cand_tok=cand, cand_logp=logp, workspace=ws8)
+        B.spec_verify(cand, rot[i % n_rot], accept_len=acc, best_cand=best, next_tok=nxt, workspace=vws)
+
+    for i in range(3):
+        step8(i)
+    torch.cuda.synchronize()
+    v0.record(stream)
+    for i in range(prof_steps):
+        step8(i)
+    v1.record(stream)
+    torch.cuda.synchronize()
+    fp8_step_ms = v0.elapsed_time(v1) / prof_steps
+    assert B.spec_poll_error(ws8) == 0
+    B.spec_detach_fp8_heads(h)
+
     if rank != 0:
         if dist is not None:
             dist.destroy_process_group()
@@ -441,6 +461,8 @@ def main():
         "head_at_BK_rows": {"rows": bk_rows, "us": round(bk_ms * 1e3, 2), "what": "spec_head_topk: head GEMM + merge",
                             "TFLOP/s": round(2.0 * bk_rows * cfg.d_inner * V / (bk_ms * 1e-3) / 1e12, 1),
                             "frac_of_burst": round(2.0 * bk_rows * cfg.d_inner * V / (bk_ms * 1e-3) / 1e12 / peaks["bf16_tflops"], 3)},
+        "step_with_e4m3_heads": {"ms_per_step": round(fp8_step_ms, 5), "value": shard.whole_job_rate(Bn, world, fp8_step_ms * 1e-3),
+                                 "what": "optional mode: e4m3 head copies on the weight-bound levels, short list re-scored in bf16"},
         "kernel_us": kernels, "kernel_us_note": "separate-kernel form bracketed by events (adds 2-3 us per kernel); "
                                                 "the timed step launches the next level's projection with the head",
         "cpu_baseline": cpu,
