@@ -32,6 +32,14 @@ METRIC = "draft+verify sequences/sec"
 UNIT = "sequences/s"
 
 
+# DRAM bytes (read + write) per launch from the ncu captures summarised under profiles/ (taken with the
+# kernels as they are in this tree; set to None when a kernel changes until it is captured again)
+NCU_TRAFFIC_BYTES = {
+    ("llama2-13b", "head_gemm_384_rows"): 279.3e6,     # profiles/gemm_tc_kernel_head_llama2-13b.md
+    ("llama2-13b", "verify_stream"): 135.2e6,          # profiles/verify_stream_kernel_llama2-13b.md
+}
+
+
 def load_peaks():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(path):
@@ -416,7 +424,8 @@ def main():
         ach = flops / (head_ms * 1e-3) / 1e12
         roof = {"kernel": f"gemm_tc_kernel (vocabulary head, level {n - 1}: {rows_last} x {cfg.d_inner} x {V})",
                 "bound": "tensor", "achieved": ach, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
-                "frac": ach / peaks["bf16_tflops"], "traffic": None, "peak_source": peaks["source"] + " burst",
+                "frac": ach / peaks["bf16_tflops"], "traffic": NCU_TRAFFIC_BYTES.get((cfg.name, f"head_gemm_{rows_last}_rows")),
+                "peak_source": peaks["source"] + " burst",
                 "frac_of_sustained": ach / peaks["bf16_tflops_sustained"]}
     else:
         ach = w_bytes / (head_ms * 1e-3) / 1e9
@@ -425,7 +434,8 @@ def main():
                 "frac": ach / peaks["hbm_gbs"], "traffic": None, "peak_source": peaks["source"]}
     v_gbs = logits_bytes / (verify_ms * 1e-3) / 1e9
     roof_verify = {"kernel": "verify_stream_kernel + verify_accept_kernel", "bound": "hbm", "achieved": v_gbs,
-                   "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": v_gbs / peaks["hbm_gbs"], "traffic": None,
+                   "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": v_gbs / peaks["hbm_gbs"],
+                   "traffic": NCU_TRAFFIC_BYTES.get((cfg.name, "verify_stream")),
                    "us": round(verify_ms * 1e3, 2), "bytes": logits_bytes,
                    "early_exit_form_us": round(verify_early_ms * 1e3, 2)}
     # heads below the ridge are weight-bandwidth bound: report their HBM fraction too
