@@ -263,9 +263,21 @@ def test_draft_fp8_heads_full_size(B, name, seqs):
     B.spec_attach_fp8_heads(h)
     got_tok, got_lp, ws = B.spec_draft(h, ctx.cuda(), tok.cuda(), cfg.topk, cfg.K)
     assert B.spec_poll_error(ws) == 0
-    same = (ref_tok == got_tok).all(dim=2).all(dim=1)
-    assert same.float().mean().item() >= 0.75, "most sequences must give identical candidate lists"
-    assert (ref_lp[same] - got_lp[same]).abs().max().item() <= cfg.n * 5e-3
+    # The normaliser of an e4m3 level comes from approximate logits (error ~1e-3 per level), so candidates
+    # whose scores nearly coincide may swap places or, at the K-th place, be exchanged: compare what is
+    # stable - the best candidate, the candidate SET of most sequences, and the scores of shared candidates.
+    rt, gt = ref_tok.cpu().numpy(), got_tok.cpu().numpy()
+    rl, gl = ref_lp.cpu().numpy(), got_lp.cpu().numpy()
+    assert (rt[:, 0] == gt[:, 0]).all(), "the most confident candidate must not change"
+    same_set = 0
+    for b in range(cfg.B):
+        ref = {tuple(c): s for c, s in zip(rt[b].tolist(), rl[b].tolist())}
+        got = {tuple(c): s for c, s in zip(gt[b].tolist(), gl[b].tolist())}
+        shared = set(ref) & set(got)
+        assert len(shared) >= cfg.K - 2
+        assert max(abs(ref[c] - got[c]) for c in shared) <= cfg.n * 5e-3
+        same_set += len(shared) == cfg.K
+    assert same_set >= 0.8 * cfg.B
     B.spec_destroy(h)
 
 
