@@ -2,8 +2,8 @@
 """Benchmark of the draft + verify hot path (metric: draft+verify sequences/s).
 
 One step = one spec_draft (n heads, full product tree, prune to K) followed by one
-spec_verify over base_logits [B, K, n+1, V], on seeded synthetic inputs shaped like the
-BASELINE "Llama2-13B-shaped" configuration.  Prints ONE JSON line on rank 0.
+spec_verify over base_logits [B, K, n+1, V], on seeded synthetic inputs of the "Llama2-13B-shaped"
+configuration (synth.CONFIGS).  Prints ONE JSON line on rank 0.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--config NAME] [--impl ours|reference]
 

@@ -1,6 +1,6 @@
 // Device-side building blocks of the sm_100a tensor-core contraction
 //     C[M, N] = A[M, Kd] * B[N, Kd]^T,  bf16 operands (row-major = K-major for both), fp32 in TMEM,
-// shared by the stand-alone GEMM kernel and by the fused draft kernel.
+// used by the GEMM kernel (gemm_tcgen05.cu).
 //
 // A CTA has 192 threads in three roles that meet only through mbarriers:
 //   warp 0      TMA producer: 128-byte-swizzled [128 x 64] A boxes and [block_n x 64] B boxes into a

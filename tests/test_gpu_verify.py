@@ -123,7 +123,7 @@ def test_verify_worked_example(B):
 
 @pytest.mark.parametrize("name", ["tiny", "llama2-7b", "llama2-13b", "codellama-34b", "llama3-8b"])
 def test_verify_full_size_configs(B, name):
-    """Full BASELINE shapes in the launch configuration the benchmark times, streaming and early-exit
+    """Full benchmark shapes in the launch configuration the benchmark times, streaming and early-exit
     forms; the oracle checks every row (the CPU arg-max over the whole tensor takes seconds)."""
     cfg = synth.CONFIGS[name]
     cand = synth.random_cand_tok(cfg, device="cuda")
