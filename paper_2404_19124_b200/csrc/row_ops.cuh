@@ -204,18 +204,6 @@ __device__ __forceinline__ void mix_ln_gelu_row(const MixArgs &m, int r, int tid
     }
 }
 
-// Picks the register-array size for the row width; false when the row is too wide for this group size.
-template <int kThreads, int kDepth, typename Sync>
-__device__ __forceinline__ bool mix_ln_gelu_row_any(const MixArgs &m, int r, int tid, float *red) {
-    const int groups = (m.d + 8 * kThreads - 1) / (8 * kThreads);
-    if (groups <= 1) mix_ln_gelu_row<kThreads, 1, kDepth, Sync>(m, r, tid, red);
-    else if (groups <= 2) mix_ln_gelu_row<kThreads, 2, kDepth, Sync>(m, r, tid, red);
-    else if (groups <= 4) mix_ln_gelu_row<kThreads, 4, kDepth, Sync>(m, r, tid, red);
-    else if (groups <= 8) mix_ln_gelu_row<kThreads, 8, kDepth, Sync>(m, r, tid, red);
-    else return false;
-    return true;
-}
-
 // (value desc, token id asc) ordering of candidates.
 __device__ __forceinline__ bool better(float v, int i, float w, int j) { return v > w || (v == w && i < j); }
 

@@ -131,7 +131,9 @@ verify_stream_kernel(const uint4 *__restrict__ logits, long long total_vec, int 
     }
 }
 
-template <bool kBf16, bool kVector>
+// Scalar fallback for tensors whose rows are not whole 16-byte vectors (or an unaligned base): fixed
+// chunks per row, one warp per (row, chunk).
+template <bool kBf16>
 __global__ void __launch_bounds__(kArgmaxThreads)
 verify_argmax_kernel(const void *__restrict__ logits, int rows, int V, int chunk_elems, int chunks,
                      float *__restrict__ pval, int32_t *__restrict__ pidx) {
@@ -145,34 +147,13 @@ verify_argmax_kernel(const void *__restrict__ logits, int rows, int V, int chunk
     const int count = min(chunk_elems, V - begin);
     constexpr int kEsz = kBf16 ? 2 : 4;
     const char *rp = (const char *)logits + ((size_t)row * V + begin) * kEsz;
-
     float best = -INFINITY;
     int idx = kIdxNone;
-    if (kVector) {
-        constexpr int kEpv = 16 / kEsz;
-        const uint4 *vp = (const uint4 *)rp;
-        const int nvec = count / kEpv;   // exact: V and chunk_elems are multiples of kEpv on this path
-        for (int v0 = lane; v0 < nvec; v0 += 128) {
-            uint4 q[4];
-#pragma unroll
-            for (int u = 0; u < 4; ++u)
-                if (v0 + 32 * u < nvec) q[u] = ld_stream(vp + v0 + 32 * u);
-#pragma unroll
-            for (int u = 0; u < 4; ++u) {
-                if (v0 + 32 * u < nvec) {
-                    const int base = begin + (v0 + 32 * u) * kEpv;
-                    if (kBf16) consume_bf16(q[u], base, best, idx);
-                    else consume_f32(q[u], base, best, idx);
-                }
-            }
-        }
-    } else {
-        for (int i = lane; i < count; i += 32) {
-            float x = kBf16 ? bf16_bits_to_float(((const uint16_t *)rp)[i]) : ((const float *)rp)[i];
-            if (x > best) {
-                best = x;
-                idx = begin + i;
-            }
+    for (int i = lane; i < count; i += 32) {
+        const float x = kBf16 ? bf16_bits_to_float(((const uint16_t *)rp)[i]) : ((const float *)rp)[i];
+        if (x > best) {
+            best = x;
+            idx = begin + i;
         }
     }
     warp_argmax(best, idx);
@@ -399,10 +380,10 @@ int launch_verify(const int32_t *cand_tok, const void *base_logits, int dtype, i
         const long long units = (long long)plan.rows * plan.chunks;
         const unsigned grid = (unsigned)((units + kWarpsPerBlock - 1) / kWarpsPerBlock);
         if (dtype == SPEC_BF16)
-            SPEC_CUDA_TRY(launch_pdl(verify_argmax_kernel<true, false>, dim3(grid), dim3(kArgmaxThreads), 0, st,
+            SPEC_CUDA_TRY(launch_pdl(verify_argmax_kernel<true>, dim3(grid), dim3(kArgmaxThreads), 0, st,
                                      base_logits, plan.rows, V, plan.chunk_elems, plan.chunks, pval, pidx));
         else
-            SPEC_CUDA_TRY(launch_pdl(verify_argmax_kernel<false, false>, dim3(grid), dim3(kArgmaxThreads), 0, st,
+            SPEC_CUDA_TRY(launch_pdl(verify_argmax_kernel<false>, dim3(grid), dim3(kArgmaxThreads), 0, st,
                                      base_logits, plan.rows, V, plan.chunk_elems, plan.chunks, pval, pidx));
     }
     const size_t smem = sizeof(int32_t) * (size_t)K * (n + 1);
