@@ -383,6 +383,21 @@ def main():
     v1.record(stream)
     torch.cuda.synchronize()
     bk_ms = v0.elapsed_time(v1) / prof_steps
+    # the dominant kernel alone: head GEMM of the last level with its fused epilogue, at that level's row
+    # count, launched back to back on the timed stream (262 MB of weights per launch: nothing stays in L2)
+    rows_dom = cfg.nodes(n - 1)
+    Sdom = Sbk[:rows_dom].contiguous() if rows_dom <= bk_rows else (
+        torch.randn(rows_dom, cfg.d_inner, generator=torch.Generator(device=dev).manual_seed(6), device=dev) * 0.5).to(torch.bfloat16)
+    dws = torch.empty(B.spec_head_workspace_bytes(h, rows_dom, hk), dtype=torch.uint8, device=dev)
+    for i in range(3):
+        B.spec_head_partials(h, n - 1, Sdom, hk, dws)
+    torch.cuda.synchronize()
+    v0.record(stream)
+    for i in range(prof_steps):
+        B.spec_head_partials(h, n - 1, Sdom, hk, dws)
+    v1.record(stream)
+    torch.cuda.synchronize()
+    head_alone_ms = v0.elapsed_time(v1) / prof_steps
 
     # the same step with e4m3 copies of the heads attached (used by the levels of up to 128 nodes)
     B.spec_attach_fp8_heads(h)
@@ -416,7 +431,8 @@ def main():
     kernels = {nm: round(ms * 1e3, 2) for nm, ms in zip(names, kern_ms)}      # microseconds
     # dominant kernel: the vocabulary-head GEMM of the last (widest) level
     rows_last = cfg.nodes(n - 1)
-    head_ms = kern_ms[4 * (n - 1) + 2]
+    head_ms = head_alone_ms   # average launch duration of the kernel itself (the per-kernel list below brackets
+                              # every launch with events, which adds 2-3 us)
     flops = 2.0 * rows_last * cfg.d_inner * V
     w_bytes = 2.0 * V * cfg.d_inner + 2.0 * rows_last * cfg.d_inner
     ridge = peaks["bf16_tflops"] * 1e12 / (peaks["hbm_gbs"] * 1e9)

@@ -211,8 +211,13 @@ int spec_poll_error(void *workspace, void *cuda_stream);
  * spec_head_topk: the fused form used inside spec_draft: per row the topk largest logits
  *   (tok, dev int32 [rows, topk]) and their log-probabilities (logp, dev fp32 [rows, topk]);
  *   full logits are never written.  workspace >= spec_head_workspace_bytes(...).
+ * spec_head_partials: only the first of spec_head_topk's two kernels, the head GEMM with its fused
+ *   epilogue (per vocabulary tile and row: partial top-k list and (max, sum-exp) in the workspace); for
+ *   timing that kernel alone.
  */
 size_t spec_head_workspace_bytes(spec_handle_t h, int rows, int topk);
+int spec_head_partials(spec_handle_t h, int level, const void *states, int rows, int topk, void *workspace,
+                       size_t workspace_bytes, void *cuda_stream);
 int spec_head_logits(spec_handle_t h, int level, const void *states /*dev bf16 [rows, d_inner]*/, int rows,
                      float *logits, void *cuda_stream);
 int spec_head_topk(spec_handle_t h, int level, const void *states, int rows, int topk, int32_t *tok, float *logp,

@@ -27,6 +27,7 @@ EXPORTS = [
     "spec_draft_workspace_bytes", "spec_draft_layout", "spec_draft", "spec_verify_workspace_bytes", "spec_verify",
     "spec_profile_read", "spec_poll_error", "spec_head_workspace_bytes", "spec_head_logits", "spec_head_topk",
     "spec_verify_static", "spec_verify_early", "spec_quantize_head", "spec_set_head_fp8",
+    "spec_head_partials",
 ]
 
 if not os.path.exists(LIB_PATH):
@@ -83,6 +84,7 @@ _lib.spec_profile_read.argtypes = [C.c_void_p, C.POINTER(C.c_float), C.c_int, C.
 _lib.spec_head_workspace_bytes.restype = C.c_size_t
 _lib.spec_head_workspace_bytes.argtypes = [C.c_void_p, C.c_int, C.c_int]
 _lib.spec_head_logits.argtypes = [C.c_void_p, C.c_int, C.c_void_p, C.c_int, C.c_void_p, C.c_void_p]
+_lib.spec_head_partials.argtypes = [C.c_void_p, C.c_int, C.c_void_p, C.c_int, C.c_int, C.c_void_p, C.c_size_t, C.c_void_p]
 _lib.spec_head_topk.argtypes = [C.c_void_p, C.c_int, C.c_void_p, C.c_int, C.c_int, C.c_void_p, C.c_void_p,
                                 C.c_void_p, C.c_size_t, C.c_void_p]
 
@@ -332,6 +334,15 @@ def spec_head_logits(h: SpecHandle, level: int, states: torch.Tensor, logits: Op
     _check(_lib.spec_head_logits(h.ptr, int(level), _ptr(states), rows, _ptr(logits), _stream_ptr(stream)),
            "spec_head_logits")
     return logits
+
+
+def spec_head_partials(h: SpecHandle, level: int, states: torch.Tensor, topk: int, workspace: torch.Tensor,
+                       stream: Optional[torch.cuda.Stream] = None) -> None:
+    """The head GEMM with its fused epilogue alone (first kernel of spec_head_topk); for timing."""
+    rows = states.shape[0]
+    _dev(states, torch.bfloat16, (rows, h.d_inner), "states")
+    _check(_lib.spec_head_partials(h.ptr, int(level), _ptr(states), rows, int(topk), _ptr(workspace),
+                                   workspace.numel(), _stream_ptr(stream)), "spec_head_partials")
 
 
 def spec_head_topk(h: SpecHandle, level: int, states: torch.Tensor, topk: int, tok: Optional[torch.Tensor] = None,

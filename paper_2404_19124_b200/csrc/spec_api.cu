@@ -556,9 +556,12 @@ int spec_head_logits(spec_handle_t h, int level, const void *states, int rows, f
                           nullptr, (cudaStream_t)cuda_stream);
 }
 
-int spec_head_topk(spec_handle_t h, int level, const void *states, int rows, int topk, int32_t *tok, float *logp,
-                   void *workspace, size_t workspace_bytes, void *cuda_stream) {
-    if (!h || !states || !tok || !logp || rows <= 0) return SPEC_ERR_INVALID_ARG;
+// The two kernels of the fused head; `tok` / `logp` null: the GEMM with its epilogue only, and no clearing
+// of the error word (so that back-to-back calls are kernel launches and nothing else).
+static int head_topk_impl(spec_handle_t h, int level, const void *states, int rows, int topk, int32_t *tok, float *logp,
+                          void *workspace, size_t workspace_bytes, void *cuda_stream) {
+    const bool merge = tok != nullptr;
+    if (!h || !states || rows <= 0 || (merge && !logp)) return SPEC_ERR_INVALID_ARG;
     if (level < 0 || level >= h->w.n_heads || topk < 1 || topk > SPEC_MAX_TOPK || topk > h->w.V) return SPEC_ERR_SHAPE;
     if ((uintptr_t)states & 15) return SPEC_ERR_INVALID_ARG;
     const size_t need = spec_head_workspace_bytes(h, rows, topk);
@@ -569,7 +572,7 @@ int spec_head_topk(spec_handle_t h, int level, const void *states, int rows, int
     const size_t units = (size_t)rows * n_tiles;
     char *ws = (char *)workspace;
     int32_t *err = (int32_t *)ws;
-    SPEC_CUDA_TRY(cudaMemsetAsync(err, 0, sizeof(int32_t), st));
+    if (merge) SPEC_CUDA_TRY(cudaMemsetAsync(err, 0, sizeof(int32_t), st));
     size_t off = kWsAlign;
     float *part_val = (float *)(ws + off);
     off = align_up(off + sizeof(float) * units * SPEC_MAX_TOPK, kWsAlign);
@@ -580,8 +583,19 @@ int spec_head_topk(spec_handle_t h, int level, const void *states, int rows, int
     float *logits_scratch = (float *)(ws + off);
     int rc = run_head_partials(h, states, h->w.head[level], rows, bn, topk, part_val, part_idx, part_ms,
                                logits_scratch, err, st);
-    if (rc != SPEC_OK) return rc;
+    if (rc != SPEC_OK || !merge) return rc;
     return launch_merge_expand(part_val, part_idx, part_ms, rows, n_tiles, topk, nullptr, tok, logp, st);
+}
+
+int spec_head_topk(spec_handle_t h, int level, const void *states, int rows, int topk, int32_t *tok, float *logp,
+                   void *workspace, size_t workspace_bytes, void *cuda_stream) {
+    if (!tok || !logp) return SPEC_ERR_INVALID_ARG;
+    return head_topk_impl(h, level, states, rows, topk, tok, logp, workspace, workspace_bytes, cuda_stream);
+}
+
+int spec_head_partials(spec_handle_t h, int level, const void *states, int rows, int topk, void *workspace,
+                       size_t workspace_bytes, void *cuda_stream) {
+    return head_topk_impl(h, level, states, rows, topk, nullptr, nullptr, workspace, workspace_bytes, cuda_stream);
 }
 
 }  // extern "C"
