@@ -39,8 +39,10 @@ enum spec_status {
                                  treated as zero and the call runs to completion)             */
     SPEC_ERR_TIMEOUT = 6,     /* device: a bounded wait inside a kernel ran out               */
     SPEC_ERR_NO_DEVICE = 7,   /* no CUDA device / not an sm_100 part                          */
-    SPEC_ERR_STATIC_SCRATCH = 8 /* spec_verify_static: the problem needs more scratch than the
+    SPEC_ERR_STATIC_SCRATCH = 8, /* spec_verify_static: the problem needs more scratch than the
                                  built-in array holds (SPEC_VERIFY_STATIC_SCRATCH_BYTES)      */
+    SPEC_ERR_INDEX_RANGE = 9  /* device: spec_next_ctx met best_cand outside [0, K) or accept_len
+                                 outside [0, n] (that sequence's row is written as zeros)     */
 };
 
 enum spec_dtype { SPEC_BF16 = 0, SPEC_F32 = 1 };
@@ -148,6 +150,20 @@ int spec_verify(const int32_t *cand_tok, const void *base_logits, int logits_dty
 int spec_verify_early(const int32_t *cand_tok, const void *base_logits, int logits_dtype, int B, int K, int n, int V,
                       int32_t *accept_len, int32_t *best_cand, int32_t *next_tok, void *workspace,
                       size_t workspace_bytes, void *cuda_stream);
+
+/* ---- closing the loop (Sec. 3.1: the speculator starts from the base model's latest state vector;
+ * after a verified step that is the state at the last accepted position of the best candidate) ----
+ *   base_state  dev bf16 [B, K, n+1, d_base]  the base model's state vectors at the positions whose
+ *                                             logits spec_verify looked at
+ *   best_cand, accept_len  dev int32 [B]      as written by spec_verify* earlier on the same stream
+ *   ctx_state   dev bf16 [B, d_base] (out)    ctx_state[b,:] = base_state[b, best_cand[b], accept_len[b], :]
+ *   err_word    dev int32, or NULL            receives SPEC_ERR_INDEX_RANGE if it was 0 and an index is
+ *                                             out of range (e.g. the word at offset 0 of the verify
+ *                                             workspace, which spec_poll_error reads); never cleared here
+ * Only enqueues one copy kernel on `cuda_stream`; nothing is allocated.  Rows are copied 16 bytes at a
+ * time when d_base is a multiple of 8 and both tensors are 16-byte aligned, else element by element. */
+int spec_next_ctx(const void *base_state, const int32_t *best_cand, const int32_t *accept_len, int B, int K, int n,
+                  int d_base, void *ctx_state, int32_t *err_word, void *cuda_stream);
 
 /* ---- verify without a caller-supplied workspace -----------------------------------------
  * (No counterpart in the paper: this is a packaging variant of spec_verify, same results.)

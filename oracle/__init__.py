@@ -6,6 +6,7 @@ imports nothing from them.  All arrays are numpy; bf16 tensors travel as ``uint1
 patterns so both sides read identical bytes.
 
 Paper passages restated by each routine are cited in ``spec_oracle.c``.
+``next_ctx`` (the one routine written here, in numpy) is pinned by a hand-built example in the tests.
 """
 from __future__ import annotations
 
@@ -275,6 +276,21 @@ def verify(cand_tok: np.ndarray, base_logits: np.ndarray, dtype: int, want_g: bo
     if rc != OK:
         raise OracleError(rc, "verify")
     return (acc, best, nxt, g) if want_g else (acc, best, nxt)
+
+
+def next_ctx(base_state: np.ndarray, best_cand: np.ndarray, accept_len: np.ndarray) -> np.ndarray:
+    """State vector the next draft starts from (Sec. 3.1: the speculator is fed the base model's latest
+    state; after a verified step that is the one at the last accepted position of the best candidate).
+    base_state [B, K, n+1, d] of any dtype -> [B, d].  Written as the loop it is, one sequence at a time."""
+    B, K, n1, d = base_state.shape
+    out = np.empty((B, d), base_state.dtype)
+    for b in range(B):
+        k, m = int(best_cand[b]), int(accept_len[b])
+        if not (0 <= k < K and 0 <= m < n1):
+            raise OracleError(1, "next_ctx: index out of range")
+        for i in range(d):
+            out[b, i] = base_state[b, k, m, i]
+    return out
 
 
 def num_threads() -> int:

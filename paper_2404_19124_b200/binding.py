@@ -17,7 +17,7 @@ LIB_PATH = os.path.join(_PKG, "libspec_b200.so")
 
 MAX_HEADS, MAX_TOPK, MAX_LEAVES = 8, 8, 4096
 (SPEC_OK, SPEC_ERR_INVALID_ARG, SPEC_ERR_SHAPE, SPEC_ERR_WORKSPACE, SPEC_ERR_CUDA, SPEC_ERR_TOKEN_RANGE,
- SPEC_ERR_TIMEOUT, SPEC_ERR_NO_DEVICE, SPEC_ERR_STATIC_SCRATCH) = range(9)
+ SPEC_ERR_TIMEOUT, SPEC_ERR_NO_DEVICE, SPEC_ERR_STATIC_SCRATCH, SPEC_ERR_INDEX_RANGE) = range(10)
 SPEC_VERIFY_STATIC_SCRATCH_BYTES = 1 << 20
 SPEC_BF16, SPEC_F32 = 0, 1
 SPEC_OPT_GEMM_IMPL, SPEC_OPT_HEAD_BLOCK_N, SPEC_OPT_PROJ_BLOCK_N, SPEC_OPT_PROFILE, SPEC_OPT_FP8_MAX_ROWS = 0, 1, 2, 3, 4
@@ -27,7 +27,7 @@ EXPORTS = [
     "spec_draft_workspace_bytes", "spec_draft_layout", "spec_draft", "spec_verify_workspace_bytes", "spec_verify",
     "spec_profile_read", "spec_poll_error", "spec_head_workspace_bytes", "spec_head_logits", "spec_head_topk",
     "spec_verify_static", "spec_verify_early", "spec_quantize_head", "spec_set_head_fp8",
-    "spec_head_partials",
+    "spec_head_partials", "spec_next_ctx",
 ]
 
 if not os.path.exists(LIB_PATH):
@@ -77,6 +77,8 @@ _lib.spec_verify.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_int, 
 _lib.spec_verify_static.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_int, C.c_int, C.c_int,
                                     C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
 _lib.spec_verify_early.argtypes = _lib.spec_verify.argtypes
+_lib.spec_next_ctx.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_int, C.c_int, C.c_void_p,
+                                C.c_void_p, C.c_void_p]
 _lib.spec_quantize_head.argtypes = [C.c_void_p, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p]
 _lib.spec_set_head_fp8.argtypes = [C.c_void_p, C.c_int, C.c_void_p, C.c_void_p]
 _lib.spec_poll_error.argtypes = [C.c_void_p, C.c_void_p]
@@ -285,6 +287,25 @@ def spec_verify_static(cand_tok: torch.Tensor, base_logits: torch.Tensor, accept
     with torch.cuda.device(cand_tok.device):
         _check(_lib.spec_verify_static(_ptr(cand_tok), _ptr(base_logits), dt, B, K, n, V, _ptr(accept_len),
                                        _ptr(best_cand), _ptr(next_tok), _stream_ptr(stream)), "spec_verify_static")
+
+
+def spec_next_ctx(base_state: torch.Tensor, best_cand: torch.Tensor, accept_len: torch.Tensor,
+                  ctx_state: Optional[torch.Tensor] = None, err_workspace: Optional[torch.Tensor] = None,
+                  stream: Optional[torch.cuda.Stream] = None) -> torch.Tensor:
+    """ctx_state[b] = base_state[b, best_cand[b], accept_len[b]]: the state the next spec_draft starts from.
+    `err_workspace` (e.g. the verify workspace) receives SPEC_ERR_INDEX_RANGE at offset 0 on a bad index."""
+    B, K, n1, d = base_state.shape
+    _dev(base_state, torch.bfloat16, name="base_state")
+    _dev(best_cand, torch.int32, (B,), "best_cand")
+    _dev(accept_len, torch.int32, (B,), "accept_len")
+    if ctx_state is None:
+        ctx_state = torch.empty((B, d), dtype=torch.bfloat16, device=base_state.device)
+    _dev(ctx_state, torch.bfloat16, (B, d), "ctx_state")
+    with torch.cuda.device(base_state.device):
+        _check(_lib.spec_next_ctx(_ptr(base_state), _ptr(best_cand), _ptr(accept_len), B, K, n1 - 1, d, _ptr(ctx_state),
+                                  _ptr(err_workspace) if err_workspace is not None else None, _stream_ptr(stream)),
+               "spec_next_ctx")
+    return ctx_state
 
 
 def spec_attach_fp8_heads(h: SpecHandle, levels: Optional[Sequence[int]] = None,

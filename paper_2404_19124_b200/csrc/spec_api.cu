@@ -197,6 +197,7 @@ const char *spec_status_str(int s) {
         case SPEC_ERR_TIMEOUT: return "bounded wait inside a kernel ran out";
         case SPEC_ERR_NO_DEVICE: return "no usable CUDA device";
         case SPEC_ERR_STATIC_SCRATCH: return "problem needs more scratch than the library's built-in array holds";
+        case SPEC_ERR_INDEX_RANGE: return "device: best_cand or accept_len out of range in spec_next_ctx";
         default: return "unknown status";
     }
 }

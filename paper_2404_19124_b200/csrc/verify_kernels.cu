@@ -417,6 +417,53 @@ int launch_verify_early(const int32_t *cand_tok, const void *base_logits, int dt
 
 }  // namespace spec
 
+// ---- spec_next_ctx: the state vector the next draft starts from (Sec. 3.1) ----------------------
+namespace spec {
+namespace {
+
+// One CTA per sequence copies base_state[b, best_cand[b], accept_len[b], :] to ctx_state[b, :].  The two
+// indices come from the verify kernels earlier in the stream, hence the dependency wait before they are read.
+__global__ void __launch_bounds__(128)
+next_ctx_kernel(const uint16_t *__restrict__ base_state, const int32_t *__restrict__ best_cand,
+                const int32_t *__restrict__ accept_len, int K, int n, int d, int vec_ok,
+                uint16_t *__restrict__ ctx_state, int32_t *err) {
+    griddep_launch();
+    griddep_wait();
+    const int b = blockIdx.x;
+    const int k = best_cand[b], m = accept_len[b];
+    uint16_t *dst = ctx_state + (size_t)b * d;
+    if (k < 0 || k >= K || m < 0 || m > n) {   // never read outside the tensor: the row becomes zero
+        if (threadIdx.x == 0) report_error(err, SPEC_ERR_INDEX_RANGE);
+        for (int i = threadIdx.x; i < d; i += blockDim.x) dst[i] = 0;
+        return;
+    }
+    const uint16_t *src = base_state + (((size_t)b * K + k) * (n + 1) + m) * d;
+    if (vec_ok) {
+        const uint4 *s4 = reinterpret_cast<const uint4 *>(src);
+        uint4 *d4 = reinterpret_cast<uint4 *>(dst);
+        for (int i = threadIdx.x; i < d / 8; i += blockDim.x) d4[i] = s4[i];
+    } else {
+        for (int i = threadIdx.x; i < d; i += blockDim.x) dst[i] = src[i];
+    }
+}
+
+}  // namespace
+}  // namespace spec
+
+extern "C" int spec_next_ctx(const void *base_state, const int32_t *best_cand, const int32_t *accept_len, int B, int K,
+                             int n, int d_base, void *ctx_state, int32_t *err_word, void *cuda_stream) {
+    using namespace spec;
+    if (!base_state || !best_cand || !accept_len || !ctx_state) return SPEC_ERR_INVALID_ARG;
+    if (B <= 0 || K <= 0 || n <= 0 || d_base <= 0) return SPEC_ERR_INVALID_ARG;
+    if (((uintptr_t)base_state % 2) != 0 || ((uintptr_t)ctx_state % 2) != 0) return SPEC_ERR_INVALID_ARG;
+    if (err_word && ((uintptr_t)err_word % 4) != 0) return SPEC_ERR_INVALID_ARG;
+    const int vec_ok = (d_base % 8 == 0) && ((uintptr_t)base_state % 16) == 0 && ((uintptr_t)ctx_state % 16) == 0;
+    SPEC_CUDA_TRY(launch_pdl(next_ctx_kernel, dim3((unsigned)B), dim3(128), 0, (cudaStream_t)cuda_stream,
+                             (const uint16_t *)base_state, best_cand, accept_len, K, n, d_base, vec_ok,
+                             (uint16_t *)ctx_state, err_word));
+    return SPEC_OK;
+}
+
 // ---- spec_verify_static: the verify scratch lives in the library's own device image ------------
 // For hosts that cannot give the library a workspace (all device memory already committed to their
 // own pools, or no allocation allowed where this runs).  Inside host code the array's name is only a

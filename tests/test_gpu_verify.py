@@ -5,7 +5,7 @@ import torch
 
 import oracle
 from paper_2404_19124_b200 import synth
-from helpers import ws_view
+from helpers import small_cfg, to_oracle_weights, weights_to_cuda, ws_view
 
 pytestmark = pytest.mark.gpu
 
@@ -154,3 +154,68 @@ def test_verify_argument_errors(B):
     with pytest.raises(B.SpecError) as e:
         B.spec_verify(cand, logits, workspace=small)
     assert e.value.status == B.SPEC_ERR_WORKSPACE
+
+
+@pytest.mark.parametrize("B_,K,n,d", [(1, 1, 1, 8), (3, 5, 3, 40), (16, 8, 3, 5120), (4, 7, 2, 13), (64, 16, 4, 4096)])
+def test_next_ctx_matches_the_oracle(B, B_, K, n, d):
+    g = torch.Generator().manual_seed(B_ * 131 + d)
+    base = torch.randn(B_, K, n + 1, d, generator=g).to(torch.bfloat16)
+    best = torch.randint(0, K, (B_,), generator=g, dtype=torch.int64).to(torch.int32)
+    acc = torch.randint(0, n + 1, (B_,), generator=g, dtype=torch.int64).to(torch.int32)
+    want = oracle.next_ctx(synth.bf16_bits(base), best.numpy(), acc.numpy())
+    err = torch.zeros(64, dtype=torch.int32, device="cuda")
+    got = B.spec_next_ctx(base.cuda(), best.cuda(), acc.cuda(), err_workspace=err)
+    assert np.array_equal(synth.bf16_bits(got.cpu()), want)
+    assert int(err[0]) == 0
+    # an unaligned view of the same data takes the element-wise path
+    if d % 8 == 0:
+        flat = torch.empty(base.numel() + 1, dtype=torch.bfloat16, device="cuda")
+        flat[1:] = base.cuda().flatten()
+        got2 = B.spec_next_ctx(flat[1:].view(B_, K, n + 1, d), best.cuda(), acc.cuda())
+        assert np.array_equal(synth.bf16_bits(got2.cpu()), want)
+
+
+def test_next_ctx_reports_bad_indices_and_writes_zeros(B):
+    B_, K, n, d = 3, 4, 2, 16
+    base = torch.ones(B_, K, n + 1, d, dtype=torch.bfloat16, device="cuda")
+    best = torch.tensor([0, K, 1], dtype=torch.int32, device="cuda")       # K is one past the end
+    acc = torch.tensor([n, 0, n + 1], dtype=torch.int32, device="cuda")    # n + 1 too
+    err = torch.zeros(64, dtype=torch.int32, device="cuda")
+    out = B.spec_next_ctx(base, best, acc, err_workspace=err)
+    assert int(err[0]) == B.SPEC_ERR_INDEX_RANGE
+    assert out.float().cpu().tolist() == [[1.0] * d, [0.0] * d, [0.0] * d]
+
+
+def test_draft_verify_next_ctx_close_the_loop(B):
+    """Three decode steps chained on the device: draft -> verify -> next_ctx -> draft, no host round trip
+    between the calls; each step's results equal the oracle's run on the same inputs."""
+    cfg = small_cfg(d_base=64, d_inner=64, V=520, topk=(3, 2, 2), K=5, B=4, seed=77)
+    sw = synth.make_weights(cfg)
+    ow, gw = to_oracle_weights(sw), weights_to_cuda(sw)
+    ctx, tok = synth.make_draft_inputs(cfg)
+    h = B.spec_create(gw)
+    ctx_d, tok_d = ctx.cuda(), tok.cuda()
+    gen = torch.Generator().manual_seed(5)
+    for step in range(3):
+        cand, logp, dws = B.spec_draft(h, ctx_d, tok_d, cfg.topk, cfg.K)
+        logits = torch.randn(cfg.B, cfg.K, cfg.n + 1, cfg.V, generator=gen).to(torch.bfloat16)
+        hidden = torch.randn(cfg.B, cfg.K, cfg.n + 1, cfg.d_base, generator=gen).to(torch.bfloat16)
+        c = cand.cpu()
+        for b in range(cfg.B):                       # make some candidates partly right
+            for k in range(cfg.K):
+                for j in range((b + k + step) % (cfg.n + 1)):
+                    logits[b, k, j, int(c[b, k, j])] = 30.0
+        acc, best, nxt, vws = B.spec_verify(cand, logits.cuda())
+        nctx = B.spec_next_ctx(hidden.cuda(), best, acc, err_workspace=vws)
+        assert B.spec_poll_error(dws) == 0 and B.spec_poll_error(vws) == 0
+        # oracle on the same inputs
+        o_cand, o_logp = oracle.draft(ow, synth.bf16_bits(ctx_d.cpu()), tok_d.cpu().numpy(), cfg.topk, cfg.K)[:2]
+        assert np.array_equal(c.numpy(), o_cand)
+        o_acc, o_best, o_nxt = oracle.verify(o_cand, synth.bf16_bits(logits), oracle.BF16)
+        assert np.array_equal(acc.cpu().numpy(), o_acc) and np.array_equal(best.cpu().numpy(), o_best)
+        assert np.array_equal(nxt.cpu().numpy(), o_nxt)
+        o_ctx = oracle.next_ctx(synth.bf16_bits(hidden), o_best, o_acc)
+        assert np.array_equal(synth.bf16_bits(nctx.cpu()), o_ctx)
+        assert int(acc.max()) > 0
+        ctx_d, tok_d = nctx, nxt
+    B.spec_destroy(h)

@@ -378,3 +378,25 @@ def test_mix_weights_follow_the_variance_rule():
         a, b = synth.mix_weights(n, 4096 ** -0.5)
         assert abs(a ** (2 * n) - 0.5) < 1e-12
         assert abs(a * a + (b * 4096 ** -0.5) ** 2 - 1.0) < 1e-12
+
+
+def test_next_ctx_hand_built_example():
+    """Sec. 3.1: the next draft starts from the base model's state at the last accepted position of the
+    best candidate.  Entry (b, k, j, i) of the tensor is the number b k j i read in base 10, so every
+    expected value below can be checked by eye."""
+    B, K, n, d = 2, 3, 2, 4
+    base = np.empty((B, K, n + 1, d), np.int64)
+    for b in range(B):
+        for k in range(K):
+            for j in range(n + 1):
+                for i in range(d):
+                    base[b, k, j, i] = 1000 * b + 100 * k + 10 * j + i
+    out = oracle.next_ctx(base, best_cand=np.array([2, 0]), accept_len=np.array([1, 2]))
+    assert out.tolist() == [[210, 211, 212, 213], [1020, 1021, 1022, 1023]]
+    # nothing accepted: the state at position 0 (the one that produced the bonus token)
+    assert oracle.next_ctx(base, np.array([1, 1]), np.array([0, 0])).tolist() == [[100, 101, 102, 103],
+                                                                                 [1100, 1101, 1102, 1103]]
+    with pytest.raises(oracle.OracleError):
+        oracle.next_ctx(base, np.array([3, 0]), np.array([0, 0]))
+    with pytest.raises(oracle.OracleError):
+        oracle.next_ctx(base, np.array([0, 0]), np.array([0, 3]))
