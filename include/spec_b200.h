@@ -115,7 +115,9 @@ int spec_set_option(spec_handle_t h, int option, int value);
  *   topk       host int32 [n_heads], 1 <= topk[l] <= SPEC_MAX_TOPK, prod <= SPEC_MAX_LEAVES
  *   K          1 <= K <= prod topk
  *   cand_tok   dev int32 [B, K, n_heads] (out), cand_logp dev fp32 [B, K] (out)
- *   workspace  dev, 256-byte aligned, >= spec_draft_workspace_bytes(...)
+ *   workspace  dev, 256-byte aligned, >= spec_draft_workspace_bytes(...).  Need not be zeroed: the
+ *              first kernel of the call clears the header (error word at byte 0, one int32
+ *              counter per sequence from byte 256 on).
  */
 size_t spec_draft_workspace_bytes(spec_handle_t h, int B, const int32_t *topk, int K);
 int spec_draft_layout(spec_handle_t h, int B, const int32_t *topk, int K, spec_draft_layout_t *out /*host*/);

@@ -76,11 +76,23 @@ __global__ void __launch_bounds__(kRowThreads) mix_ln_gelu_wide_kernel(MixArgs m
         m.S_out[(size_t)r * d + i] = (uint16_t)float_to_bf16_bits(gelu_erf((h_s[i] - mean) * rstd * m.gamma[i] + m.beta[i]));
 }
 
+// First kernel of a draft: clears the workspace header (error word, per-sequence counters).  A kernel
+// rather than a memset so that the projection launched behind it may already set itself up and fetch
+// weights; like every kernel here it first waits for whatever precedes it in the stream.
+__global__ void __launch_bounds__(256) draft_init_kernel(int32_t *hdr, int words) {
+    griddep_launch();
+    griddep_wait();
+    for (int i = threadIdx.x; i < words; i += blockDim.x) hdr[i] = 0;
+}
+
 __global__ void __launch_bounds__(kMergeThreads) merge_expand_kernel(MergeArgs g) {
+    extern __shared__ LeafKey merge_keys[];   // [Lpad] when the prune is folded in, else nothing
     __shared__ Scratch sc;
+    __shared__ int last_of_sequence;
     griddep_launch();
     griddep_wait();
     merge_expand_row<kMergeThreads, BlockSync>(g, blockIdx.x, threadIdx.x, &sc);
+    prune_if_last<kMergeThreads, BlockSync>(g, blockIdx.x, threadIdx.x, merge_keys, &last_of_sequence);
 }
 
 __global__ void __launch_bounds__(kRowThreads)
@@ -112,12 +124,14 @@ int launch_mix_ln_gelu(const MixArgs &m, int rows, cudaStream_t st) {
     return SPEC_OK;
 }
 
-int launch_merge_expand(const float *part_val, const int32_t *part_idx, const float *part_ms, int rows, int n_tiles,
-                        int topk, const float *score_in, int32_t *tok_out, float *score_out, cudaStream_t st) {
-    MergeArgs g{};
-    g.part_val = part_val; g.part_idx = part_idx; g.part_ms = part_ms;
-    g.n_tiles = n_tiles; g.topk = topk; g.score_in = score_in; g.tok_out = tok_out; g.score_out = score_out;
-    SPEC_CUDA_TRY(launch_pdl(merge_expand_kernel, dim3(rows), dim3(kMergeThreads), 0, st, g));
+int launch_draft_init(int32_t *hdr, int words, cudaStream_t st) {
+    SPEC_CUDA_TRY(launch_pdl(draft_init_kernel, dim3(1), dim3(256), 0, st, hdr, words));
+    return SPEC_OK;
+}
+
+int launch_merge_expand(const MergeArgs &g, int rows, cudaStream_t st) {
+    const size_t smem = g.seq_done ? sizeof(LeafKey) * (size_t)g.Lpad : 0;
+    SPEC_CUDA_TRY(launch_pdl(merge_expand_kernel, dim3(rows), dim3(kMergeThreads), smem, st, g));
     return SPEC_OK;
 }
 

@@ -65,8 +65,10 @@ struct RescoreArgs {
 
 // One CTA per row.
 __global__ void __launch_bounds__(kRescoreThreads) merge_rescore_kernel(RescoreArgs a) {
+    extern __shared__ LeafKey rescore_keys[];   // [Lpad] when the prune is folded in, else nothing
     __shared__ Scratch sc;
     __shared__ float exact[kShortList];
+    __shared__ int last_of_sequence;
     griddep_launch();
     griddep_wait();
     const int r = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -127,6 +129,7 @@ __global__ void __launch_bounds__(kRescoreThreads) merge_rescore_kernel(RescoreA
             }
         }
     }
+    prune_if_last<kRescoreThreads, BlockSync>(a.merge, r, tid, rescore_keys, &last_of_sequence);
 }
 
 }  // namespace
@@ -145,7 +148,8 @@ int launch_merge_rescore(const MergeArgs &g, const void *W, const void *S, int r
     a.S = (const uint16_t *)S;
     a.d = d;
     a.V = V;
-    SPEC_CUDA_TRY(launch_pdl(merge_rescore_kernel, dim3(rows), dim3(kRescoreThreads), 0, st, a));
+    const size_t smem = g.seq_done ? sizeof(LeafKey) * (size_t)g.Lpad : 0;
+    SPEC_CUDA_TRY(launch_pdl(merge_rescore_kernel, dim3(rows), dim3(kRescoreThreads), smem, st, a));
     return SPEC_OK;
 }
 

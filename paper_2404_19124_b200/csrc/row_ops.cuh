@@ -444,5 +444,24 @@ __device__ __forceinline__ void prune_sequence(const float *leaf_score, const Pr
         emit_candidate(pa, L, K, cand_tok, cand_logp, b, k, keys[k].score, keys[k].leaf);
 }
 
+// Prune folded into the kernel that writes the last level.  Every row's CTA makes its children visible
+// (fence), then counts itself in for its sequence; the CTA that brings the count to rows_per_seq sees all
+// of the sequence's leaves and prunes it.  No CTA ever waits for another.  `flag`: one shared int.
+template <int kThreads, typename Sync>
+__device__ __forceinline__ void prune_if_last(const MergeArgs &g, int r, int tid, LeafKey *keys, int *flag) {
+    if (g.seq_done == nullptr) return;
+    const int b = r / g.rows_per_seq;
+    __threadfence();
+    Sync::sync();
+    if (tid == 0) {
+        __threadfence();
+        *flag = (atomicAdd(g.seq_done + b, 1) == g.rows_per_seq - 1) ? 1 : 0;
+    }
+    Sync::sync();
+    if (*flag == 0) return;
+    __threadfence();
+    prune_sequence<kThreads, Sync>(g.score_out, g.prune, g.L, g.Lpad, g.K, g.cand_tok, g.cand_logp, b, tid, keys);
+}
+
 }  // namespace rows
 }  // namespace spec

@@ -57,6 +57,8 @@ struct DraftPlan {
     int proj_block_n[SPEC_MAX_HEADS];
     int proj_splits[SPEC_MAX_HEADS];   // > 0: swapped split-K projection (few parent rows); 0: plain
     bool use_fp8[SPEC_MAX_HEADS];      // the level's head runs on the e4m3 copy of its weights
+    size_t seq_done;                   // byte offset of the per-sequence counters of the folded prune
+    int header_words;                  // int32 words cleared at the start of a draft
 };
 
 int head_block_n_for(const spec_handle_s *h, int rows) {
@@ -102,8 +104,11 @@ int make_draft_plan(const spec_handle_s *h, int B, const int32_t *topk, int K, D
     p->L = (int)leaves;
 
     spec_draft_layout_t &y = p->lay;
-    size_t off = kWsAlign;   // error word lives at offset 0
+    // header: the error word at offset 0, one int32 counter per sequence from byte 256 on
     y.error_word = 0;
+    p->seq_done = kWsAlign;
+    p->header_words = (int)(kWsAlign / sizeof(int32_t)) + B;
+    size_t off = align_up(kWsAlign + sizeof(int32_t) * (size_t)B, kWsAlign);
     for (int l = 1; l <= p->n; ++l) {
         y.tok[l] = off;
         off = align_up(off + sizeof(int32_t) * (size_t)p->N[l], kWsAlign);
@@ -339,7 +344,8 @@ int spec_draft(spec_handle_t h, const void *ctx_state, const int32_t *last_tok, 
     const spec_weights_t &w = h->w;
     char *ws = (char *)workspace;
     int32_t *err = (int32_t *)(ws + p.lay.error_word);
-    SPEC_CUDA_TRY(cudaMemsetAsync(err, 0, sizeof(int32_t), st));
+    rc = launch_draft_init(err, p.header_words, st);
+    if (rc != SPEC_OK) return rc;
 
     int nev = 0;
     h->prof_count = 0;
@@ -379,6 +385,13 @@ int spec_draft(spec_handle_t h, const void *ctx_state, const int32_t *last_tok, 
         }
         return c;
     };
+    PruneArgs pa{};
+    pa.n = p.n;
+    for (int l = 0; l < p.n; ++l) {
+        pa.tok[l] = (const int32_t *)(ws + p.lay.tok[l + 1]);
+        pa.topk[l] = topk[l];
+    }
+    const bool fold_prune = !h->profile;
     bool proj_done = false;   // the projection of the level about to start ran with the previous head
     for (int l = 0; l < p.n; ++l) {
         const int rows = p.N[l];
@@ -448,33 +461,40 @@ int spec_draft(spec_handle_t h, const void *ctx_state, const int32_t *last_tok, 
         }
         if (rc != SPEC_OK) return rc;
         SPEC_PROF_MARK();
-        // fold the partials, branch: children (token, cumulative score) of every node
+        // fold the partials, branch: children (token, cumulative score) of every node.  On the last
+        // level the CTA that completes a sequence's leaves also prunes it (one kernel less on the
+        // critical path; with per-kernel profiling the prune stays a launch of its own).
+        MergeArgs g{};
+        g.part_val = part_val; g.part_idx = part_idx; g.part_ms = part_ms;
+        g.n_tiles = p.lay.n_tiles[l]; g.topk = topk[l];
+        g.score_in = score_l;
+        g.tok_out = (int32_t *)(ws + p.lay.tok[l + 1]);
+        g.score_out = (float *)(ws + p.lay.score[l + 1]);
+        if (l == p.n - 1 && fold_prune) {
+            g.seq_done = (int32_t *)(ws + p.seq_done);
+            g.rows_per_seq = rows / B;
+            g.L = p.L; g.K = K;
+            g.Lpad = 2;
+            while (g.Lpad < p.L) g.Lpad <<= 1;
+            g.cand_tok = cand_tok; g.cand_logp = cand_logp;
+            g.prune = pa;
+        }
         if (fp8) {
             // short list by approximate logit, exact re-scoring from the bf16 weights, then the children
-            MergeArgs g{};
-            g.part_val = part_val; g.part_idx = part_idx; g.part_ms = part_ms;
-            g.n_tiles = p.lay.n_tiles[l]; g.topk = topk[l]; g.list_len = SPEC_MAX_TOPK;
-            g.score_in = score_l;
-            g.tok_out = (int32_t *)(ws + p.lay.tok[l + 1]);
-            g.score_out = (float *)(ws + p.lay.score[l + 1]);
+            g.list_len = SPEC_MAX_TOPK;
             rc = launch_merge_rescore(g, w.head[l], S, rows, w.d_inner, w.V, st);
         } else {
-            rc = launch_merge_expand(part_val, part_idx, part_ms, rows, p.lay.n_tiles[l], topk[l], score_l,
-                                     (int32_t *)(ws + p.lay.tok[l + 1]), (float *)(ws + p.lay.score[l + 1]), st);
+            rc = launch_merge_expand(g, rows, st);
         }
         if (rc != SPEC_OK) return rc;
         SPEC_PROF_MARK();
     }
 
-    PruneArgs pa{};
-    pa.n = p.n;
-    for (int l = 0; l < p.n; ++l) {
-        pa.tok[l] = (const int32_t *)(ws + p.lay.tok[l + 1]);
-        pa.topk[l] = topk[l];
+    if (!fold_prune) {
+        rc = launch_prune((const float *)(ws + p.lay.score[p.n]), pa, B, p.L, K, cand_tok, cand_logp, st);
+        if (rc != SPEC_OK) return rc;
+        SPEC_PROF_MARK();
     }
-    rc = launch_prune((const float *)(ws + p.lay.score[p.n]), pa, B, p.L, K, cand_tok, cand_logp, st);
-    if (rc != SPEC_OK) return rc;
-    SPEC_PROF_MARK();
 #undef SPEC_PROF_MARK
     h->prof_count = nev;
     return SPEC_OK;
@@ -585,7 +605,11 @@ static int head_topk_impl(spec_handle_t h, int level, const void *states, int ro
     int rc = run_head_partials(h, states, h->w.head[level], rows, bn, topk, part_val, part_idx, part_ms,
                                logits_scratch, err, st);
     if (rc != SPEC_OK || !merge) return rc;
-    return launch_merge_expand(part_val, part_idx, part_ms, rows, n_tiles, topk, nullptr, tok, logp, st);
+    MergeArgs g{};
+    g.part_val = part_val; g.part_idx = part_idx; g.part_ms = part_ms;
+    g.n_tiles = n_tiles; g.topk = topk;
+    g.tok_out = tok; g.score_out = logp;
+    return launch_merge_expand(g, rows, st);
 }
 
 int spec_head_topk(spec_handle_t h, int level, const void *states, int rows, int topk, int32_t *tok, float *logp,

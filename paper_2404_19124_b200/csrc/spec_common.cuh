@@ -139,6 +139,12 @@ struct MixArgs {
     int32_t *err;
 };
 
+struct PruneArgs {
+    const int32_t *tok[SPEC_MAX_HEADS]; // tok[l]: tokens of level l+1 nodes
+    int32_t topk[SPEC_MAX_HEADS];
+    int n;
+};
+
 struct MergeArgs {
     const float *part_val;     // [rows, n_tiles, SPEC_MAX_TOPK] (first `topk` of each list valid, any order)
     const int32_t *part_idx;   // same shape
@@ -148,6 +154,14 @@ struct MergeArgs {
     const float *score_in;     // [rows] or null (score 0)
     int32_t *tok_out;          // [rows, topk]
     float *score_out;          // [rows, topk]
+    // Last level only (seq_done != null): the CTA whose row completes a sequence's leaves prunes that
+    // sequence in the same launch, so no separate prune kernel waits behind this one.
+    int32_t *seq_done;         // [B] rows finished per sequence, zero before the launch
+    int rows_per_seq;          // rows of this level per sequence
+    int L, Lpad, K;            // leaves per sequence, L padded to a power of two >= 2, candidates kept
+    int32_t *cand_tok;         // [B, K, n]
+    float *cand_logp;          // [B, K]
+    PruneArgs prune;
 };
 
 // e4m3 copy of a bf16 matrix: Q [rows, d] bytes and one fp32 scale per row (fp8.cuh).
@@ -155,14 +169,9 @@ int launch_quantize_rows(const void *X, int rows, int d, void *Q, float *scale, 
 // merge of approximate partial lists + exact re-scoring of the short list + expansion (fp8_kernels.cu)
 int launch_merge_rescore(const MergeArgs &g, const void *W, const void *S, int rows, int d, int V, cudaStream_t st);
 
+int launch_draft_init(int32_t *hdr, int words, cudaStream_t st);
 int launch_mix_ln_gelu(const MixArgs &m, int rows, cudaStream_t st);
-int launch_merge_expand(const float *part_val, const int32_t *part_idx, const float *part_ms, int rows, int n_tiles,
-                        int topk, const float *score_in, int32_t *tok_out, float *score_out, cudaStream_t st);
-struct PruneArgs {
-    const int32_t *tok[SPEC_MAX_HEADS]; // tok[l]: tokens of level l+1 nodes
-    int32_t topk[SPEC_MAX_HEADS];
-    int n;
-};
+int launch_merge_expand(const MergeArgs &g, int rows, cudaStream_t st);
 int launch_prune(const float *leaf_score, const PruneArgs &pa, int B, int L, int K, int32_t *cand_tok,
                  float *cand_logp, cudaStream_t st);
 
