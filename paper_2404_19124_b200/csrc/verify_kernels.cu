@@ -166,10 +166,13 @@ verify_argmax_kernel(const void *__restrict__ logits, int rows, int V, int chunk
 __global__ void __launch_bounds__(128)
 verify_accept_kernel(const int32_t *__restrict__ cand_tok, const float *__restrict__ pval,
                      const int32_t *__restrict__ pidx, int K, int n, int slots, int vpr, int vec_per_warp,
-                     int32_t *__restrict__ g_out,
+                     int32_t *g_out, int g_in_smem,
                      int32_t *__restrict__ accept_len, int32_t *__restrict__ best_cand,
                      int32_t *__restrict__ next_tok, int32_t *err) {
-    extern __shared__ int32_t g_s[];   // [K * (n + 1)]
+    // The sequence's arg-max table is re-read by other threads for the prefix match: from shared memory
+    // when it fits the default 48 KB, otherwise from the copy in g_out this CTA has just written (global
+    // writes of a CTA are visible to its own threads after the barrier).
+    extern __shared__ int32_t g_s[];   // [K * (n + 1)] if g_in_smem
     __shared__ unsigned int key_s;
     const int b = blockIdx.x, rows_b = K * (n + 1);
     griddep_launch();
@@ -194,13 +197,14 @@ verify_accept_kernel(const int32_t *__restrict__ cand_tok, const float *__restri
                 arg = pidx[u0 + c];
             }
         }
-        g_s[r] = arg;
+        if (g_in_smem) g_s[r] = arg;
         g_out[(size_t)b * rows_b + r] = arg;
     }
     __syncthreads();
+    const int32_t *gtab = g_in_smem ? g_s : g_out + (size_t)b * rows_b;
     for (int k = threadIdx.x; k < K; k += blockDim.x) {
         const int32_t *c = cand_tok + ((size_t)b * K + k) * n;
-        const int32_t *gk = g_s + k * (n + 1);
+        const int32_t *gk = gtab + k * (n + 1);
         int m = 0;
         while (m < n && c[m] == gk[m]) ++m;
         // longest prefix first, then the lowest candidate index
@@ -211,7 +215,7 @@ verify_accept_kernel(const int32_t *__restrict__ cand_tok, const float *__restri
         const int m = (int)(key_s >> 16), k = 0xffff - (int)(key_s & 0xffffu);
         accept_len[b] = m;
         best_cand[b] = k;
-        next_tok[b] = g_s[k * (n + 1) + m];
+        next_tok[b] = gtab[k * (n + 1) + m];
     }
 }
 
@@ -386,10 +390,12 @@ int launch_verify(const int32_t *cand_tok, const void *base_logits, int dtype, i
             SPEC_CUDA_TRY(launch_pdl(verify_argmax_kernel<false>, dim3(grid), dim3(kArgmaxThreads), 0, st,
                                      base_logits, plan.rows, V, plan.chunk_elems, plan.chunks, pval, pidx));
     }
-    const size_t smem = sizeof(int32_t) * (size_t)K * (n + 1);
+    size_t smem = sizeof(int32_t) * (size_t)K * (n + 1);
+    const int g_in_smem = smem <= 40 * 1024;
+    if (!g_in_smem) smem = 0;
     SPEC_CUDA_TRY(launch_pdl(verify_accept_kernel, dim3(B), dim3(128), smem, st, cand_tok, (const float *)pval,
                              (const int32_t *)pidx, K, n, stream ? plan.slots : plan.chunks, plan.vpr, vec_per_warp,
-                             g, accept_len, best_cand, next_tok, err));
+                             g, g_in_smem, accept_len, best_cand, next_tok, err));
     return SPEC_OK;
 }
 

@@ -371,3 +371,29 @@ def test_draft_then_verify_chain_and_graph_replay(B):
     for got, want in zip((cand, logp, acc, best, nxt), ref):
         assert torch.equal(got, want)
     B.spec_destroy(h)
+
+
+@pytest.mark.parametrize("topk,K,fp8", [((8, 8, 8), 100, False), ((8, 8, 8), 512, False), ((8, 8, 8, 8), 300, False),
+                                        ((8, 8, 8, 8), 4096, False), ((4, 4, 4, 5), 320, True)])
+def test_draft_many_leaves_up_to_the_limit(B, topk, K, fp8):
+    """More than 256 leaves per sequence (the sorted prune instead of the ranked one), up to
+    SPEC_MAX_LEAVES = 4096 with K = every leaf."""
+    cfg = small_cfg(d_base=48, d_inner=64, V=96, topk=topk, K=K, B=2, seed=sum(topk) + K)
+    chk = _draft_and_check(B, cfg, fp8=fp8)
+    assert chk.exact + chk.tolerated == cfg.B
+
+
+def test_draft_refuses_more_leaves_than_the_limit(B):
+    cfg = small_cfg(d_base=48, d_inner=64, V=96, topk=(8, 8, 8, 8, 2), K=4, B=1, seed=1)   # 8192 leaves
+    sw, ow, gw = _setup(cfg)
+    h = B.spec_create(gw)
+    ctx, tok = synth.make_draft_inputs(cfg)
+    assert B.spec_draft_workspace_bytes(h, 1, cfg.topk, 4) == 0
+    with pytest.raises(B.SpecError) as e:
+        B.spec_draft(h, ctx.cuda(), tok.cuda(), cfg.topk, 4)
+    assert e.value.status == B.SPEC_ERR_SHAPE
+    assert B.spec_draft_workspace_bytes(h, 1, (8, 8, 8, 8, 1), 4096) > 0       # exactly at the limit
+    with pytest.raises(B.SpecError) as e:                                       # K beyond the leaves
+        B.spec_draft(h, ctx.cuda(), tok.cuda(), (8, 8, 8, 8, 1), 4097)
+    assert e.value.status == B.SPEC_ERR_SHAPE
+    B.spec_destroy(h)

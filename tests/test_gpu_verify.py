@@ -219,3 +219,32 @@ def test_draft_verify_next_ctx_close_the_loop(B):
         assert int(acc.max()) > 0
         ctx_d, tok_d = nctx, nxt
     B.spec_destroy(h)
+
+
+@pytest.mark.parametrize("K,n", [(4096, 2), (1536, 7), (12288 // 33, 32)])
+def test_verify_at_the_row_limit(B, K, n):
+    """K (n + 1) = 12288 rows per sequence (or the largest K below it) is the documented limit."""
+    Bn, V = 2, 40
+    g = torch.Generator().manual_seed(K + n)
+    logits = torch.randn(Bn, K, n + 1, V, generator=g).to(torch.bfloat16)
+    cand = torch.randint(0, V, (Bn, K, n), generator=g, dtype=torch.int64).to(torch.int32)
+    am = logits.to(torch.float32).argmax(-1)
+    cand[0, K - 1] = am[0, K - 1, :n].to(torch.int32)        # the last candidate of sequence 0 is fully right
+    cand[1, K // 2, : n // 2 + 1] = am[1, K // 2, : n // 2 + 1].to(torch.int32)
+    want = oracle.verify(cand.numpy(), synth.bf16_bits(logits), oracle.BF16)
+    for early in (False, True):
+        acc, best, nxt, _ = B.spec_verify(cand.cuda(), logits.cuda(), early_exit=early)
+        for a, w in zip((acc, best, nxt), want):
+            assert np.array_equal(a.cpu().numpy(), w)
+    assert int(want[0][0]) == n
+
+
+def test_verify_refuses_more_rows_than_the_limit(B):
+    K, n, V = 4097, 2, 8                                       # 12291 rows per sequence
+    logits = torch.zeros(1, K, n + 1, V, dtype=torch.bfloat16, device="cuda")
+    cand = torch.zeros(1, K, n, dtype=torch.int32, device="cuda")
+    ws = torch.empty(1 << 22, dtype=torch.uint8, device="cuda")
+    outs = [torch.empty(1, dtype=torch.int32, device="cuda") for _ in range(3)]
+    with pytest.raises(B.SpecError) as e:
+        B.spec_verify(cand, logits, accept_len=outs[0], best_cand=outs[1], next_tok=outs[2], workspace=ws)
+    assert e.value.status == B.SPEC_ERR_SHAPE
