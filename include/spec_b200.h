@@ -204,7 +204,8 @@ int spec_verify_static(const int32_t *cand_tok, const void *base_logits, int log
  * in e4m3 (tensor cores, fp32 accumulation), keeps the 16 tokens with the best APPROXIMATE logits
  * per node, recomputes those 16 logits exactly from the bf16 weights and states, and branches
  * to the top-k of the exact values; only the softmax normaliser comes from the approximate
- * logits (its error is of order 1e-3 in log-probability).  d_inner must be a multiple of 16.
+ * logits (its error is of order 1e-3 in log-probability).  d_inner must be a multiple of 16;
+ * with d_inner > 16384 the attached copies are ignored and every level runs in bf16.
  *   spec_quantize_head  fills q_out (dev, V * d_inner bytes, 16-byte aligned) and scale_out
  *                       (dev fp32 [V]) from head `level`'s bf16 weights on `cuda_stream`
  *   spec_set_head_fp8   attaches such a pair to the handle (caller-owned, must outlive the calls

@@ -137,7 +137,9 @@ int make_draft_plan(const spec_handle_s *h, int B, const int32_t *topk, int K, D
     off = align_up(off + sizeof(float) * max_proj_floats, kWsAlign);
     int max_fp8_rows = 0;
     for (int l = 0; l < p->n; ++l) {
-        p->use_fp8[l] = h->gemm_impl == 0 && !h->profile && h->head8[l] != nullptr && p->N[l] <= h->fp8_max_rows;
+        // (the mix kernel for rows wider than 16384 elements keeps them in shared memory and has no e4m3 output)
+        p->use_fp8[l] = h->gemm_impl == 0 && !h->profile && h->head8[l] != nullptr && p->N[l] <= h->fp8_max_rows &&
+                        w.d_inner <= 16384;
         if (p->use_fp8[l] && p->N[l] > max_fp8_rows) max_fp8_rows = p->N[l];
     }
     y.state8 = off;

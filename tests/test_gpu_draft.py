@@ -397,3 +397,13 @@ def test_draft_refuses_more_leaves_than_the_limit(B):
         B.spec_draft(h, ctx.cuda(), tok.cuda(), (8, 8, 8, 8, 1), 4097)
     assert e.value.status == B.SPEC_ERR_SHAPE
     B.spec_destroy(h)
+
+
+@pytest.mark.parametrize("d,fp8", [(4104, False), (5120, False), (16384, False), (16448, False),
+                                   (5120, True), (16384, True), (16448, True)])
+def test_draft_wide_states(B, d, fp8):
+    """State widths beyond the benchmark shapes: each range of d_inner has its own mix + LayerNorm + GELU
+    kernel (rows kept in registers up to 16384 elements, in shared memory beyond)."""
+    cfg = small_cfg(d_base=64, d_inner=d, V=264, topk=(2, 2), K=3, B=2, seed=d % 97)
+    chk = _draft_and_check(B, cfg, check_levels=not fp8, fp8=fp8)
+    assert chk.exact + chk.tolerated == cfg.B
