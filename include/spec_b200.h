@@ -196,6 +196,42 @@ int spec_next_ctx(const void *base_state, const int32_t *best_cand, const int32_
 int spec_verify_static(const int32_t *cand_tok, const void *base_logits, int logits_dtype, int B, int K, int n,
                        int V, int32_t *accept_len, int32_t *best_cand, int32_t *next_tok, void *cuda_stream);
 
+/* ---- vocabulary-parallel heads (optional; Sec. 3.1: nearly all of the speculator's parameters sit in
+ * the vocabulary-sized matrices, which is what a small batch spends its time reading) ---------------
+ * n_ranks processes, one GPU each, split every head matrix by vocabulary rows: rank g holds rows
+ * [vocab_offset_g, vocab_offset_g + head_rows_g) of each head (the shards tile [0, V) without overlap),
+ * everything else (embeddings with all V rows, projections, LayerNorm) is replicated.  A draft becomes,
+ * per level l = 0 .. n_heads-1,
+ *     spec_draft_vp_local(level l)   projection, mix, the head on this rank's rows, and this rank's
+ *                                    lists written to slot `rank` of the exchange region
+ *     all-gather of the slots        done by the CALLER with whatever collective it has (NCCL, peer
+ *                                    copies): afterwards every rank holds all n_ranks slots
+ *     spec_draft_vp_merge(level l)   folds the slots into the level's children; at the last level also
+ *                                    prunes to the K candidates
+ * and every rank ends with the same cand_tok / cand_logp as spec_draft on unsplit weights (token sets and
+ * order identical; log-probabilities equal up to the rounding of a two-stage log-sum-exp).
+ *   spec_set_vocab_shard     declares that the head[] matrices given to spec_create hold `head_rows` rows
+ *                            starting at token `vocab_offset` (weights.V stays the full vocabulary).
+ *                            n_ranks <= 8, n_ranks * topk[l] <= 64.  On such a handle spec_draft, the
+ *                            spec_head_* calls and the e4m3 option are refused / ignored.  n_ranks = 1
+ *                            (offset 0, all rows) makes the handle an ordinary one again.
+ *   spec_draft_vp_exchange   byte offset of slot 0 in the workspace and the size of one slot at `level`;
+ *                            slot g lies at offset + g * slot_bytes.  A slot is fp32 [N_l, topk[l]] logits,
+ *                            int32 [N_l, topk[l]] token ids, fp32 [N_l] log-sum-exp over the shard, padded
+ *                            to 256 bytes.
+ *   spec_draft_vp_local / _merge  arguments as spec_draft; the same B, topk, K and workspace for every
+ *                            step of one draft (workspace size: spec_draft_workspace_bytes on the sharded
+ *                            handle).  cand_tok / cand_logp are written by the merge of the last level
+ *                            only and may be NULL before.  All calls only enqueue work on `cuda_stream`.
+ */
+int spec_set_vocab_shard(spec_handle_t h, int rank, int n_ranks, int vocab_offset, int head_rows);
+int spec_draft_vp_exchange(spec_handle_t h, int B, const int32_t *topk, int K, int level, uint64_t *offset /*host*/,
+                           uint64_t *slot_bytes /*host*/);
+int spec_draft_vp_local(spec_handle_t h, int level, const void *ctx_state, const int32_t *last_tok, int B,
+                        const int32_t *topk, int K, void *workspace, size_t workspace_bytes, void *cuda_stream);
+int spec_draft_vp_merge(spec_handle_t h, int level, int B, const int32_t *topk, int K, int32_t *cand_tok,
+                        float *cand_logp, void *workspace, size_t workspace_bytes, void *cuda_stream);
+
 /* ---- e4m3 copy of a vocabulary head (optional) ---------------------------------------------
  * (The paper runs everything in 16 bits; this is an implementation option for the heads whose
  * cost is reading the weights: levels with few nodes.)  A head's bf16 matrix [V, d_inner] can be

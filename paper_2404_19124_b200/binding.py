@@ -8,7 +8,7 @@ from __future__ import annotations
 
 import ctypes as C
 import os
-from typing import List, Optional, Sequence
+from typing import Tuple, List, Optional, Sequence
 
 import torch
 
@@ -28,6 +28,7 @@ EXPORTS = [
     "spec_profile_read", "spec_poll_error", "spec_head_workspace_bytes", "spec_head_logits", "spec_head_topk",
     "spec_verify_static", "spec_verify_early", "spec_quantize_head", "spec_set_head_fp8",
     "spec_head_partials", "spec_next_ctx",
+    "spec_set_vocab_shard", "spec_draft_vp_exchange", "spec_draft_vp_local", "spec_draft_vp_merge",
 ]
 
 if not os.path.exists(LIB_PATH):
@@ -77,6 +78,13 @@ _lib.spec_verify.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_int, 
 _lib.spec_verify_static.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_int, C.c_int, C.c_int,
                                     C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
 _lib.spec_verify_early.argtypes = _lib.spec_verify.argtypes
+_lib.spec_set_vocab_shard.argtypes = [C.c_void_p, C.c_int, C.c_int, C.c_int, C.c_int]
+_lib.spec_draft_vp_exchange.argtypes = [C.c_void_p, C.c_int, C.POINTER(C.c_int32), C.c_int, C.c_int,
+                                        C.POINTER(C.c_uint64), C.POINTER(C.c_uint64)]
+_lib.spec_draft_vp_local.argtypes = [C.c_void_p, C.c_int, C.c_void_p, C.c_void_p, C.c_int, C.POINTER(C.c_int32), C.c_int,
+                                     C.c_void_p, C.c_size_t, C.c_void_p]
+_lib.spec_draft_vp_merge.argtypes = [C.c_void_p, C.c_int, C.c_int, C.POINTER(C.c_int32), C.c_int, C.c_void_p, C.c_void_p,
+                                     C.c_void_p, C.c_size_t, C.c_void_p]
 _lib.spec_next_ctx.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_int, C.c_int, C.c_void_p,
                                 C.c_void_p, C.c_void_p]
 _lib.spec_quantize_head.argtypes = [C.c_void_p, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p]
@@ -138,11 +146,16 @@ class SpecHandle:
 
     def __init__(self, emb: List[torch.Tensor], proj: List[torch.Tensor], ln_gamma: List[torch.Tensor],
                  ln_beta: List[torch.Tensor], head: List[torch.Tensor], state_weight: float, emb_weight: float,
-                 ln_eps: float = 1e-5):
+                 ln_eps: float = 1e-5, vocab_shard: Optional[Tuple[int, int, int]] = None):
+        """vocab_shard = (rank, n_ranks, vocab_offset): the head tensors hold only the vocabulary rows
+        [vocab_offset, vocab_offset + head[l].shape[0]) (spec_set_vocab_shard); emb keeps all V rows."""
         n = len(head)
         if not (1 <= n <= MAX_HEADS) or not all(len(x) == n for x in (emb, proj, ln_gamma, ln_beta)):
             raise ValueError("need the same number (1..8) of emb / proj / ln_gamma / ln_beta / head tensors")
-        V, d_inner = head[0].shape
+        head_rows, d_inner = head[0].shape
+        V = emb[0].shape[0]
+        if head_rows != V and vocab_shard is None:
+            raise ValueError("head tensors with fewer rows than the embeddings need vocab_shard=(rank, n_ranks, offset)")
         d_base = proj[0].shape[1]
         w = SpecWeightsC()
         w.n_heads, w.V, w.d_base, w.d_inner = n, V, d_base, d_inner
@@ -152,7 +165,7 @@ class SpecHandle:
             w.proj[l] = _dev(proj[l], torch.bfloat16, (d_inner, d_in), f"proj[{l}]").data_ptr()
             w.ln_gamma[l] = _dev(ln_gamma[l], torch.float32, (d_inner,), f"ln_gamma[{l}]").data_ptr()
             w.ln_beta[l] = _dev(ln_beta[l], torch.float32, (d_inner,), f"ln_beta[{l}]").data_ptr()
-            w.head[l] = _dev(head[l], torch.bfloat16, (V, d_inner), f"head[{l}]").data_ptr()
+            w.head[l] = _dev(head[l], torch.bfloat16, (head_rows, d_inner), f"head[{l}]").data_ptr()
         w.state_weight, w.emb_weight, w.ln_eps = state_weight, emb_weight, ln_eps
         self._keep = (emb, proj, ln_gamma, ln_beta, head)
         self.n_heads, self.V, self.d_base, self.d_inner = n, V, d_base, d_inner
@@ -160,6 +173,11 @@ class SpecHandle:
         self._h = C.c_void_p()
         with torch.cuda.device(self.device):
             _check(_lib.spec_create(C.byref(self._h), C.byref(w)), "spec_create")
+        self.vp_rank, self.vp_ranks = 0, 1
+        if vocab_shard is not None:
+            rank, n_ranks, offset = (int(x) for x in vocab_shard)
+            _check(_lib.spec_set_vocab_shard(self._h, rank, n_ranks, offset, int(head_rows)), "spec_set_vocab_shard")
+            self.vp_rank, self.vp_ranks = rank, n_ranks
 
     def close(self) -> None:
         if getattr(self, "_h", None) and self._h.value:
@@ -177,11 +195,11 @@ class SpecHandle:
         return self._h
 
 
-def spec_create(weights) -> SpecHandle:
+def spec_create(weights, vocab_shard: Optional[Tuple[int, int, int]] = None) -> SpecHandle:
     """`weights`: an object with emb / proj / ln_gamma / ln_beta / head tensor lists (CUDA) and the scalars
-    state_weight, emb_weight, ln_eps (e.g. synth.SpecWeights moved to the GPU)."""
+    state_weight, emb_weight, ln_eps (e.g. synth.SpecWeights moved to the GPU).  vocab_shard: see SpecHandle."""
     return SpecHandle(weights.emb, weights.proj, weights.ln_gamma, weights.ln_beta, weights.head,
-                      weights.state_weight, weights.emb_weight, weights.ln_eps)
+                      weights.state_weight, weights.emb_weight, weights.ln_eps, vocab_shard=vocab_shard)
 
 
 def spec_destroy(h: SpecHandle) -> None:
@@ -225,6 +243,42 @@ def spec_draft(h: SpecHandle, ctx_state: torch.Tensor, last_tok: torch.Tensor, t
     _check(_lib.spec_draft(h.ptr, _ptr(ctx_state), _ptr(last_tok), B, _topk_arr(topk), int(K), _ptr(cand_tok),
                            _ptr(cand_logp), _ptr(workspace), workspace.numel(), _stream_ptr(stream)), "spec_draft")
     return cand_tok, cand_logp, workspace
+
+
+def spec_set_vocab_shard(h: SpecHandle, rank: int, n_ranks: int, vocab_offset: int, head_rows: int) -> None:
+    _check(_lib.spec_set_vocab_shard(h.ptr, int(rank), int(n_ranks), int(vocab_offset), int(head_rows)),
+           "spec_set_vocab_shard")
+    h.vp_rank, h.vp_ranks = int(rank), int(n_ranks)
+
+
+def spec_draft_vp_exchange(h: SpecHandle, B: int, topk: Sequence[int], K: int, level: int) -> Tuple[int, int]:
+    """(byte offset of slot 0 in the draft workspace, bytes of one rank's slot) at `level`."""
+    off, sz = C.c_uint64(), C.c_uint64()
+    _check(_lib.spec_draft_vp_exchange(h.ptr, int(B), _topk_arr(topk), int(K), int(level), C.byref(off), C.byref(sz)),
+           "spec_draft_vp_exchange")
+    return int(off.value), int(sz.value)
+
+
+def spec_draft_vp_local(h: SpecHandle, level: int, ctx_state: torch.Tensor, last_tok: torch.Tensor,
+                        topk: Sequence[int], K: int, workspace: torch.Tensor,
+                        stream: Optional[torch.cuda.Stream] = None) -> None:
+    B = ctx_state.shape[0]
+    _dev(ctx_state, torch.bfloat16, (B, h.d_base), "ctx_state")
+    _dev(last_tok, torch.int32, (B,), "last_tok")
+    _check(_lib.spec_draft_vp_local(h.ptr, int(level), _ptr(ctx_state), _ptr(last_tok), B, _topk_arr(topk), int(K),
+                                    _ptr(workspace), workspace.numel(), _stream_ptr(stream)), "spec_draft_vp_local")
+
+
+def spec_draft_vp_merge(h: SpecHandle, level: int, B: int, topk: Sequence[int], K: int, workspace: torch.Tensor,
+                        cand_tok: Optional[torch.Tensor] = None, cand_logp: Optional[torch.Tensor] = None,
+                        stream: Optional[torch.cuda.Stream] = None) -> None:
+    if cand_tok is not None:
+        _dev(cand_tok, torch.int32, (B, K, h.n_heads), "cand_tok")
+        _dev(cand_logp, torch.float32, (B, K), "cand_logp")
+    _check(_lib.spec_draft_vp_merge(h.ptr, int(level), int(B), _topk_arr(topk), int(K),
+                                    _ptr(cand_tok) if cand_tok is not None else None,
+                                    _ptr(cand_logp) if cand_logp is not None else None,
+                                    _ptr(workspace), workspace.numel(), _stream_ptr(stream)), "spec_draft_vp_merge")
 
 
 def spec_verify_workspace_bytes(B: int, K: int, n: int, V: int, logits_dtype: int) -> int:

@@ -95,6 +95,65 @@ __global__ void __launch_bounds__(kMergeThreads) merge_expand_kernel(MergeArgs g
     prune_if_last<kMergeThreads, BlockSync>(g, blockIdx.x, threadIdx.x, merge_keys, &last_of_sequence);
 }
 
+// Vocabulary-parallel head: one warp per row folds the n_ranks raw lists (see launch_merge_shards).
+// Lane i owns entries i and i + 32 of the row's n_ranks * topk <= 64 candidates.
+constexpr int kShardRowsPerCta = 4;
+__global__ void __launch_bounds__(32 * kShardRowsPerCta)
+merge_shards_kernel(const char *slots, size_t slot_bytes, int n_ranks, int rows, int topk,
+                    const float *__restrict__ score_in, int32_t *__restrict__ tok_out, float *__restrict__ score_out) {
+    griddep_launch();
+    griddep_wait();
+    const int lane = threadIdx.x & 31;
+    const int r = blockIdx.x * kShardRowsPerCta + (threadIdx.x >> 5);
+    if (r >= rows) return;
+    const int n_cand = n_ranks * topk;
+    float v[2];
+    int id[2];
+#pragma unroll
+    for (int q = 0; q < 2; ++q) {
+        const int c = lane + 32 * q;
+        v[q] = -INFINITY;
+        id[q] = 0x7fffffff;
+        if (c < n_cand) {
+            const int g = c / topk, j = c - g * topk;
+            const char *slot = slots + (size_t)g * slot_bytes;
+            const float *val = reinterpret_cast<const float *>(slot);
+            const int32_t *tok = reinterpret_cast<const int32_t *>(slot + sizeof(float) * (size_t)rows * topk);
+            v[q] = __ldcg(val + (size_t)r * topk + j);
+            id[q] = __ldcg(tok + (size_t)r * topk + j);
+        }
+    }
+    // log-sum-exp over the whole vocabulary from the shards' values, lane g holding shard g
+    float l = -INFINITY;
+    if (lane < n_ranks) {
+        const char *slot = slots + (size_t)lane * slot_bytes;
+        l = __ldcg(reinterpret_cast<const float *>(slot + 2 * sizeof(float) * (size_t)rows * topk) + r);
+    }
+    float m = l;
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, off));
+    float e = (lane < n_ranks && l > -INFINITY) ? expf(l - m) : 0.0f;
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) e += __shfl_xor_sync(0xffffffffu, e, off);
+    const float lse = m + logf(e);
+    const float base = score_in ? __ldcg(score_in + r) : 0.0f;
+    for (int j = 0; j < topk; ++j) {
+        // the lane's better entry, then the warp's best: (value desc, token id asc)
+        const int mine = better(v[1], id[1], v[0], id[0]) ? 1 : 0;
+        const uint32_t key = float_key(v[mine]);
+        const uint32_t bk = __reduce_max_sync(0xffffffffu, key);
+        const uint32_t bi = __reduce_min_sync(0xffffffffu, key == bk ? (uint32_t)id[mine] : 0xffffffffu);
+        if (lane == 0) {
+            tok_out[(size_t)r * topk + j] = (int)bi;
+            score_out[(size_t)r * topk + j] = base + (key_float(bk) - lse);
+        }
+        if (key == bk && (uint32_t)id[mine] == bi) {   // token ids are unique across shards: one owner
+            v[mine] = -INFINITY;
+            id[mine] = 0x7fffffff;
+        }
+    }
+}
+
 __global__ void __launch_bounds__(kRowThreads)
 prune_kernel(const float *leaf_score, PruneArgs pa, int L, int Lpad, int K, int32_t *cand_tok, float *cand_logp) {
     extern __shared__ LeafKey keys[];   // [Lpad]
@@ -132,6 +191,15 @@ int launch_draft_init(int32_t *hdr, int words, cudaStream_t st) {
 int launch_merge_expand(const MergeArgs &g, int rows, cudaStream_t st) {
     const size_t smem = g.seq_done ? sizeof(LeafKey) * (size_t)g.Lpad : 0;
     SPEC_CUDA_TRY(launch_pdl(merge_expand_kernel, dim3(rows), dim3(kMergeThreads), smem, st, g));
+    return SPEC_OK;
+}
+
+int launch_merge_shards(const void *slots, size_t slot_bytes, int n_ranks, int rows, int topk, const float *score_in,
+                        int32_t *tok_out, float *score_out, cudaStream_t st) {
+    if (n_ranks < 1 || n_ranks > 32 || n_ranks * topk > 64) return SPEC_ERR_SHAPE;
+    const int grid = (rows + kShardRowsPerCta - 1) / kShardRowsPerCta;
+    SPEC_CUDA_TRY(launch_pdl(merge_shards_kernel, dim3(grid), dim3(32 * kShardRowsPerCta), 0, st, (const char *)slots,
+                             slot_bytes, n_ranks, rows, topk, score_in, tok_out, score_out));
     return SPEC_OK;
 }
 

@@ -116,18 +116,19 @@ int make_tmap(CUtensorMap *map, const void *base, uint64_t rows, uint64_t cols, 
 // tiles fill the SMs (tiles / (waves * SMs)); among near-equal fills the widest tile wins
 // because it re-reads A least often.
 int choose_block_n(int M, int N, int num_sm, bool prefer_wide) {
+    // Cost model: the launch takes (tiles per CTA) x (cost of one tile), a tile costing its width plus a fixed
+    // part (operand A, commit and epilogue hand-over) worth 96 columns when the MMAs are the bound (more than
+    // one 128-row tile) and 32 when the weight stream is.  Ties go to the wider tile.
     const int m_tiles = (M + kBlockM - 1) / kBlockM;
+    const int fixed = prefer_wide ? 96 : 32;
     int best = 32;
-    double best_score = -1.0;
+    long long best_cost = -1;
     for (int bn = 32; bn <= 256; bn += 32) {
         const long long tiles = (long long)m_tiles * ((N + bn - 1) / bn);
         const long long waves = (tiles + num_sm - 1) / num_sm;
-        double fill = (double)tiles / (double)(waves * num_sm);
-        // wasted columns of the ragged last tile count against the candidate
-        fill *= (double)N / (double)(((N + bn - 1) / bn) * (long long)bn);
-        const double score = fill + (prefer_wide ? 0.0004 : 0.0001) * bn;
-        if (score > best_score + 1e-9) {
-            best_score = score;
+        const long long cost = waves * (bn + fixed);
+        if (best_cost < 0 || cost <= best_cost) {
+            best_cost = cost;
             best = bn;
         }
     }

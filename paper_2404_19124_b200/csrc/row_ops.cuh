@@ -372,12 +372,13 @@ __device__ __forceinline__ void merge_select(const MergeArgs &g, int r, int tid,
 // The row's top-k tokens and log-probabilities become its children.
 template <int kThreads, typename Sync>
 __device__ __forceinline__ void merge_expand_row(const MergeArgs &g, int r, int tid, Scratch *sc) {
-    const float base = (tid < g.topk && g.score_in) ? __ldcg(g.score_in + r) : 0.0f;   // in flight during the merge
+    const float base = (tid < g.topk && g.score_in && !g.lse_out) ? __ldcg(g.score_in + r) : 0.0f;   // in flight during the merge
     merge_select<kThreads, Sync>(g, r, tid, sc, g.topk);
     if (tid < g.topk) {
         g.tok_out[(size_t)r * g.topk + tid] = sc->out_id[tid];
-        g.score_out[(size_t)r * g.topk + tid] = base + (sc->out_val[tid] - sc->lse);
+        g.score_out[(size_t)r * g.topk + tid] = g.lse_out ? sc->out_val[tid] : base + (sc->out_val[tid] - sc->lse);
     }
+    if (g.lse_out != nullptr && tid == 0) g.lse_out[r] = sc->lse;
 }
 
 struct LeafKey {

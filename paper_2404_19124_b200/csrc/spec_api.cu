@@ -38,6 +38,8 @@ struct spec_handle_s {
     int fp8_max_rows;                      // SPEC_OPT_FP8_MAX_ROWS
     const void *head8[SPEC_MAX_HEADS];     // e4m3 copies of the heads (caller-owned), null: none
     const float *head8_scale[SPEC_MAX_HEADS];
+    int vp_rank, vp_ranks;                 // vocabulary-parallel heads: this handle's shard (vp_ranks 1: none)
+    int vocab_offset, head_rows;           // its head matrices hold vocabulary rows [vocab_offset, +head_rows)
     int prof_count;                        // events recorded by the last profiled draft
     cudaEvent_t prof_ev[kMaxProfEvents];   // created when profiling is switched on
 };
@@ -59,11 +61,13 @@ struct DraftPlan {
     bool use_fp8[SPEC_MAX_HEADS];      // the level's head runs on the e4m3 copy of its weights
     size_t seq_done;                   // byte offset of the per-sequence counters of the folded prune
     int header_words;                  // int32 words cleared at the start of a draft
+    size_t xchg;                       // vocabulary-parallel heads: byte offset of the rank slots
+    size_t slot_bytes[SPEC_MAX_HEADS]; // bytes of one rank's slot at each level
 };
 
 int head_block_n_for(const spec_handle_s *h, int rows) {
     if (h->head_block_n > 0) return h->head_block_n;
-    return choose_block_n(rows, h->w.V, num_sms(), rows > 128);
+    return choose_block_n(rows, h->head_rows, num_sms(), rows > 128);
 }
 
 int proj_block_n_for(const spec_handle_s *h, int rows) {
@@ -94,7 +98,7 @@ int make_draft_plan(const spec_handle_s *h, int B, const int32_t *topk, int K, D
     long long nodes = B, leaves = 1;
     p->N[0] = B;
     for (int l = 0; l < p->n; ++l) {
-        if (topk[l] < 1 || topk[l] > SPEC_MAX_TOPK || topk[l] > w.V) return SPEC_ERR_SHAPE;
+        if (topk[l] < 1 || topk[l] > SPEC_MAX_TOPK || topk[l] > h->head_rows) return SPEC_ERR_SHAPE;
         leaves *= topk[l];
         nodes *= topk[l];
         if (leaves > SPEC_MAX_LEAVES || nodes > (1ll << 24)) return SPEC_ERR_SHAPE;
@@ -109,6 +113,17 @@ int make_draft_plan(const spec_handle_s *h, int B, const int32_t *topk, int K, D
     p->seq_done = kWsAlign;
     p->header_words = (int)(kWsAlign / sizeof(int32_t)) + B;
     size_t off = align_up(kWsAlign + sizeof(int32_t) * (size_t)B, kWsAlign);
+    // vocabulary-parallel heads: one slot per rank for the lists that are exchanged after every level.  It
+    // comes first so that its offset is the same on every rank (what follows depends on the shard's size).
+    p->xchg = off;
+    if (h->vp_ranks > 1) {
+        size_t max_slot = 0;
+        for (int l = 0; l < p->n; ++l) {
+            p->slot_bytes[l] = align_up((size_t)p->N[l] * (8 * (size_t)topk[l] + 4), kWsAlign);
+            if (p->slot_bytes[l] > max_slot) max_slot = p->slot_bytes[l];
+        }
+        off = align_up(off + max_slot * h->vp_ranks, kWsAlign);
+    }
     for (int l = 1; l <= p->n; ++l) {
         y.tok[l] = off;
         off = align_up(off + sizeof(int32_t) * (size_t)p->N[l], kWsAlign);
@@ -127,7 +142,7 @@ int make_draft_plan(const spec_handle_s *h, int B, const int32_t *topk, int K, D
         if (pf > max_proj_floats) max_proj_floats = pf;
         const int bn = head_block_n_for(h, p->N[l]);
         y.block_n[l] = bn;
-        y.n_tiles[l] = (w.V + bn - 1) / bn;
+        y.n_tiles[l] = (h->head_rows + bn - 1) / bn;
         const size_t units = (size_t)p->N[l] * y.n_tiles[l];
         if (units > max_part_units) max_part_units = units;
         if (p->N[l] > max_rows) max_rows = p->N[l];
@@ -139,7 +154,7 @@ int make_draft_plan(const spec_handle_s *h, int B, const int32_t *topk, int K, D
     for (int l = 0; l < p->n; ++l) {
         // (the mix kernel for rows wider than 16384 elements keeps them in shared memory and has no e4m3 output)
         p->use_fp8[l] = h->gemm_impl == 0 && !h->profile && h->head8[l] != nullptr && p->N[l] <= h->fp8_max_rows &&
-                        w.d_inner <= 16384;
+                        w.d_inner <= 16384 && h->vp_ranks == 1;
         if (p->use_fp8[l] && p->N[l] > max_fp8_rows) max_fp8_rows = p->N[l];
     }
     y.state8 = off;
@@ -185,6 +200,61 @@ int run_head_partials(const spec_handle_s *h, const void *states, const void *Wo
     e.part_ms = part_ms;
     e.topk = topk;
     return launch_gemm_tc(states, Wout, rows, w.V, w.d_inner, block_n, e, err, st);
+}
+
+// State projection of level l as a tensor-core contraction: with few parent rows the weights take the
+// 128-row side and split-K partials are stored transposed, otherwise the plain form.
+GemmCall make_proj_call(const spec_handle_s *h, const DraftPlan &p, char *ws, const void *ctx_state, int B, int l) {
+    const spec_weights_t &w = h->w;
+    const int parent_rows = l == 0 ? B : p.N[l - 1];
+    const void *parent_states = l == 0 ? ctx_state : (const void *)(ws + p.lay.state[l - 1]);
+    GemmCall c{};
+    c.Kd = d_in_of(w, l);
+    c.epi.out = (float *)(ws + p.lay.proj);
+    c.epi.ldc = w.d_inner;
+    if (p.proj_splits[l] > 0) {
+        c.A = w.proj[l]; c.M = w.d_inner;
+        c.B = parent_states; c.N = parent_rows;
+        c.block_n = (parent_rows + 31) / 32 * 32;
+        c.epi.mode = 2;
+        c.epi.splits = p.proj_splits[l];
+        c.epi.split_stride = (size_t)parent_rows * w.d_inner;
+    } else {
+        c.A = parent_states; c.M = parent_rows;
+        c.B = w.proj[l]; c.N = w.d_inner;
+        c.block_n = p.proj_block_n[l];
+        c.epi.mode = 0;
+    }
+    return c;
+}
+
+// Arguments of the gather + mix + LayerNorm + GELU step of level l (bf16 states only).
+MixArgs make_mix_args(const spec_handle_s *h, const DraftPlan &p, char *ws, const int32_t *last_tok, int B,
+                      const int32_t *topk, int l, int32_t *err) {
+    const spec_weights_t &w = h->w;
+    const int parent_rows = l == 0 ? B : p.N[l - 1];
+    MixArgs mx{};
+    mx.P = (float *)(ws + p.lay.proj);
+    mx.p_splits = p.proj_splits[l] > 0 ? p.proj_splits[l] : 1;
+    mx.p_split_stride = (size_t)parent_rows * w.d_inner;
+    mx.emb = (const uint16_t *)w.emb[l];
+    mx.tok = l == 0 ? last_tok : (const int32_t *)(ws + p.lay.tok[l]);
+    mx.gamma = w.ln_gamma[l]; mx.beta = w.ln_beta[l];
+    mx.d = w.d_inner; mx.V = w.V; mx.parent_div = l == 0 ? 1 : topk[l - 1];
+    mx.a = w.state_weight; mx.b = w.emb_weight; mx.eps = w.ln_eps;
+    mx.S_out = (uint16_t *)(ws + p.lay.state[l]);
+    mx.err = err;
+    return mx;
+}
+
+PruneArgs make_prune_args(const DraftPlan &p, char *ws, const int32_t *topk) {
+    PruneArgs pa{};
+    pa.n = p.n;
+    for (int l = 0; l < p.n; ++l) {
+        pa.tok[l] = (const int32_t *)(ws + p.lay.tok[l + 1]);
+        pa.topk[l] = topk[l];
+    }
+    return pa;
 }
 
 }  // namespace
@@ -242,6 +312,10 @@ int spec_create(spec_handle_t *out, const spec_weights_t *w) {
     h->proj_block_n = 0;
     h->profile = 0;
     h->fp8_max_rows = 128;
+    h->vp_rank = 0;
+    h->vp_ranks = 1;
+    h->vocab_offset = 0;
+    h->head_rows = w->V;
     for (int l = 0; l < SPEC_MAX_HEADS; ++l) {
         h->head8[l] = nullptr;
         h->head8_scale[l] = nullptr;
@@ -290,7 +364,7 @@ int spec_set_option(spec_handle_t h, int option, int value) {
 }
 
 int spec_quantize_head(spec_handle_t h, int level, void *q_out, float *scale_out, void *cuda_stream) {
-    if (!h || !q_out || !scale_out) return SPEC_ERR_INVALID_ARG;
+    if (!h || !q_out || !scale_out || h->vp_ranks > 1) return SPEC_ERR_INVALID_ARG;
     if (level < 0 || level >= h->w.n_heads || h->w.d_inner % 16 != 0) return SPEC_ERR_SHAPE;
     if ((uintptr_t)q_out & 15) return SPEC_ERR_INVALID_ARG;
     return launch_quantize_rows(h->w.head[level], h->w.V, h->w.d_inner, q_out, scale_out, (cudaStream_t)cuda_stream);
@@ -337,6 +411,7 @@ int spec_draft(spec_handle_t h, const void *ctx_state, const int32_t *last_tok, 
                int32_t *cand_tok, float *cand_logp, void *workspace, size_t workspace_bytes, void *cuda_stream) {
     if (!h || !ctx_state || !last_tok || !topk || !cand_tok || !cand_logp) return SPEC_ERR_INVALID_ARG;
     if ((uintptr_t)ctx_state & 15) return SPEC_ERR_INVALID_ARG;
+    if (h->vp_ranks > 1) return SPEC_ERR_INVALID_ARG;   // a vocabulary shard: spec_draft_vp_local / _merge
     DraftPlan p;
     int rc = make_draft_plan(h, B, topk, K, &p);
     if (rc != SPEC_OK) return rc;
@@ -363,49 +438,18 @@ int spec_draft(spec_handle_t h, const void *ctx_state, const int32_t *last_tok, 
     float *part_ms = (float *)(ws + p.lay.part_ms);
     float *logits_scratch = (float *)(ws + p.lay.logits);
 
-    // state projection of level l as a tensor-core contraction: with few parent rows the weights take
-    // the 128-row side and split-K partials are stored transposed, otherwise the plain form
-    auto proj_call = [&](int l) {
-        const int parent_rows = l == 0 ? B : p.N[l - 1];
-        const void *parent_states = l == 0 ? ctx_state : (const void *)(ws + p.lay.state[l - 1]);
-        GemmCall c{};
-        c.Kd = d_in_of(w, l);
-        c.epi.out = P;
-        c.epi.ldc = w.d_inner;
-        if (p.proj_splits[l] > 0) {
-            c.A = w.proj[l]; c.M = w.d_inner;
-            c.B = parent_states; c.N = parent_rows;
-            c.block_n = (parent_rows + 31) / 32 * 32;
-            c.epi.mode = 2;
-            c.epi.splits = p.proj_splits[l];
-            c.epi.split_stride = (size_t)parent_rows * w.d_inner;
-        } else {
-            c.A = parent_states; c.M = parent_rows;
-            c.B = w.proj[l]; c.N = w.d_inner;
-            c.block_n = p.proj_block_n[l];
-            c.epi.mode = 0;
-        }
-        return c;
-    };
-    PruneArgs pa{};
-    pa.n = p.n;
-    for (int l = 0; l < p.n; ++l) {
-        pa.tok[l] = (const int32_t *)(ws + p.lay.tok[l + 1]);
-        pa.topk[l] = topk[l];
-    }
+    auto proj_call = [&](int l) { return make_proj_call(h, p, ws, ctx_state, B, l); };
+    const PruneArgs pa = make_prune_args(p, ws, topk);
     const bool fold_prune = !h->profile;
     bool proj_done = false;   // the projection of the level about to start ran with the previous head
     for (int l = 0; l < p.n; ++l) {
         const int rows = p.N[l];
         const int parent_rows = l == 0 ? B : p.N[l - 1];
         const void *parent_states = l == 0 ? ctx_state : (const void *)(ws + p.lay.state[l - 1]);
-        const int32_t *tok_l = l == 0 ? last_tok : (const int32_t *)(ws + p.lay.tok[l]);
         const float *score_l = l == 0 ? nullptr : (const float *)(ws + p.lay.score[l]);
         void *S = ws + p.lay.state[l];
         // projection of every distinct parent state: P = S_parent * Wp^T (unless it already ran in the
         // same launch as the previous level's head, see below)
-        const int splits = p.proj_splits[l];
-        const size_t split_stride = (size_t)parent_rows * w.d_inner;
         if (!proj_done) {
             if (h->gemm_impl == 0) {
                 const GemmCall c = proj_call(l);
@@ -419,12 +463,7 @@ int spec_draft(spec_handle_t h, const void *ctx_state, const int32_t *last_tok, 
         SPEC_PROF_MARK();
         // gather + mix + LayerNorm + GELU -> bf16 state of every node of this level
         const bool fp8 = p.use_fp8[l];
-        MixArgs mx{};
-        mx.P = P; mx.p_splits = splits > 0 ? splits : 1; mx.p_split_stride = split_stride;
-        mx.emb = (const uint16_t *)w.emb[l]; mx.tok = tok_l; mx.gamma = w.ln_gamma[l]; mx.beta = w.ln_beta[l];
-        mx.d = w.d_inner; mx.V = w.V; mx.parent_div = l == 0 ? 1 : topk[l - 1];
-        mx.a = w.state_weight; mx.b = w.emb_weight; mx.eps = w.ln_eps;
-        mx.S_out = (uint16_t *)S; mx.err = err;
+        MixArgs mx = make_mix_args(h, p, ws, last_tok, B, topk, l, err);
         if (fp8) {   // the head of this level reads the states as e4m3
             mx.S8_out = (uint8_t *)(ws + p.lay.state8);
             mx.s8_scale = (float *)(ws + p.lay.state8_scale);
@@ -439,7 +478,7 @@ int spec_draft(spec_handle_t h, const void *ctx_state, const int32_t *last_tok, 
         proj_done = false;
         if (h->gemm_impl == 0 && !h->profile && (l + 1 < p.n || fp8)) {
             GemmCall c[2];
-            c[0].A = S; c[0].B = w.head[l]; c[0].M = rows; c[0].N = w.V; c[0].Kd = w.d_inner;
+            c[0].A = S; c[0].B = w.head[l]; c[0].M = rows; c[0].N = h->head_rows; c[0].Kd = w.d_inner;
             c[0].block_n = p.lay.block_n[l];
             c[0].epi = GemmEpilogue{};
             c[0].epi.mode = 1;
@@ -502,6 +541,107 @@ int spec_draft(spec_handle_t h, const void *ctx_state, const int32_t *last_tok, 
     return SPEC_OK;
 }
 
+/* ---- vocabulary-parallel heads ------------------------------------------------------------------ */
+int spec_set_vocab_shard(spec_handle_t h, int rank, int n_ranks, int vocab_offset, int head_rows) {
+    if (!h) return SPEC_ERR_INVALID_ARG;
+    if (n_ranks < 1 || n_ranks > 8 || rank < 0 || rank >= n_ranks) return SPEC_ERR_INVALID_ARG;
+    if (vocab_offset < 0 || head_rows < 1 || (long long)vocab_offset + head_rows > h->w.V) return SPEC_ERR_SHAPE;
+    if (n_ranks == 1 && (vocab_offset != 0 || head_rows != h->w.V)) return SPEC_ERR_SHAPE;
+    h->vp_rank = rank;
+    h->vp_ranks = n_ranks;
+    h->vocab_offset = vocab_offset;
+    h->head_rows = head_rows;
+    return SPEC_OK;
+}
+
+int spec_draft_vp_exchange(spec_handle_t h, int B, const int32_t *topk, int K, int level, uint64_t *offset,
+                           uint64_t *slot_bytes) {
+    if (!h || !offset || !slot_bytes || h->vp_ranks < 2) return SPEC_ERR_INVALID_ARG;
+    DraftPlan p;
+    int rc = make_draft_plan(h, B, topk, K, &p);
+    if (rc != SPEC_OK) return rc;
+    if (level < 0 || level >= p.n) return SPEC_ERR_INVALID_ARG;
+    *offset = p.xchg;
+    *slot_bytes = p.slot_bytes[level];
+    return SPEC_OK;
+}
+
+int spec_draft_vp_local(spec_handle_t h, int level, const void *ctx_state, const int32_t *last_tok, int B,
+                        const int32_t *topk, int K, void *workspace, size_t workspace_bytes, void *cuda_stream) {
+    if (!h || !ctx_state || !last_tok || !topk) return SPEC_ERR_INVALID_ARG;
+    if ((uintptr_t)ctx_state & 15) return SPEC_ERR_INVALID_ARG;
+    if (h->vp_ranks < 2 || h->gemm_impl != 0) return SPEC_ERR_INVALID_ARG;
+    DraftPlan p;
+    int rc = make_draft_plan(h, B, topk, K, &p);
+    if (rc != SPEC_OK) return rc;
+    if (level < 0 || level >= p.n) return SPEC_ERR_INVALID_ARG;
+    if (!workspace || ((uintptr_t)workspace % kWsAlign) != 0 || workspace_bytes < p.lay.total_bytes)
+        return SPEC_ERR_WORKSPACE;
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    const spec_weights_t &w = h->w;
+    char *ws = (char *)workspace;
+    int32_t *err = (int32_t *)(ws + p.lay.error_word);
+    const int l = level, rows = p.N[l];
+    if (l == 0) {   // the first step of a draft clears the header and projects the context states
+        rc = launch_draft_init(err, p.header_words, st);
+        if (rc != SPEC_OK) return rc;
+        const GemmCall c = make_proj_call(h, p, ws, ctx_state, B, 0);
+        rc = launch_gemm_tc_jobs(&c, 1, err, st);
+        if (rc != SPEC_OK) return rc;
+    }
+    const MixArgs mx = make_mix_args(h, p, ws, last_tok, B, topk, l, err);
+    rc = launch_mix_ln_gelu(mx, rows, st);
+    if (rc != SPEC_OK) return rc;
+    // this rank's vocabulary rows only; token ids leave the epilogue already offset.  The next level's
+    // projection (replicated on every rank) rides in the same launch as in spec_draft.
+    GemmCall c[2];
+    c[0] = GemmCall{};
+    c[0].A = ws + p.lay.state[l]; c[0].B = w.head[l]; c[0].M = rows; c[0].N = h->head_rows; c[0].Kd = w.d_inner;
+    c[0].block_n = p.lay.block_n[l];
+    c[0].epi.mode = 1;
+    c[0].epi.part_val = (float *)(ws + p.lay.part_val);
+    c[0].epi.part_idx = (int32_t *)(ws + p.lay.part_idx);
+    c[0].epi.part_ms = (float *)(ws + p.lay.part_ms);
+    c[0].epi.topk = topk[l];
+    c[0].epi.idx_offset = h->vocab_offset;
+    const bool pair = l + 1 < p.n;
+    if (pair) c[1] = make_proj_call(h, p, ws, ctx_state, B, l + 1);
+    rc = launch_gemm_tc_jobs(c, pair ? 2 : 1, err, st);
+    if (rc != SPEC_OK) return rc;
+    // fold the tiles into this rank's slot: the shard's topk logits, their token ids, its log-sum-exp
+    char *slot = ws + p.xchg + (size_t)h->vp_rank * p.slot_bytes[l];
+    MergeArgs g{};
+    g.part_val = c[0].epi.part_val; g.part_idx = c[0].epi.part_idx; g.part_ms = c[0].epi.part_ms;
+    g.n_tiles = p.lay.n_tiles[l]; g.topk = topk[l];
+    g.score_out = (float *)slot;
+    g.tok_out = (int32_t *)(slot + sizeof(float) * (size_t)rows * topk[l]);
+    g.lse_out = (float *)(slot + 2 * sizeof(float) * (size_t)rows * topk[l]);
+    return launch_merge_expand(g, rows, st);
+}
+
+int spec_draft_vp_merge(spec_handle_t h, int level, int B, const int32_t *topk, int K, int32_t *cand_tok,
+                        float *cand_logp, void *workspace, size_t workspace_bytes, void *cuda_stream) {
+    if (!h || !topk) return SPEC_ERR_INVALID_ARG;
+    if (h->vp_ranks < 2) return SPEC_ERR_INVALID_ARG;
+    DraftPlan p;
+    int rc = make_draft_plan(h, B, topk, K, &p);
+    if (rc != SPEC_OK) return rc;
+    if (level < 0 || level >= p.n) return SPEC_ERR_INVALID_ARG;
+    const bool last = level == p.n - 1;
+    if (last && (!cand_tok || !cand_logp)) return SPEC_ERR_INVALID_ARG;
+    if (!workspace || ((uintptr_t)workspace % kWsAlign) != 0 || workspace_bytes < p.lay.total_bytes)
+        return SPEC_ERR_WORKSPACE;
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    char *ws = (char *)workspace;
+    const int l = level;
+    rc = launch_merge_shards(ws + p.xchg, p.slot_bytes[l], h->vp_ranks, p.N[l], topk[l],
+                             l == 0 ? nullptr : (const float *)(ws + p.lay.score[l]),
+                             (int32_t *)(ws + p.lay.tok[l + 1]), (float *)(ws + p.lay.score[l + 1]), st);
+    if (rc != SPEC_OK || !last) return rc;
+    return launch_prune((const float *)(ws + p.lay.score[p.n]), make_prune_args(p, ws, topk), B, p.L, K, cand_tok,
+                        cand_logp, st);
+}
+
 size_t spec_verify_workspace_bytes(int B, int K, int n, int V, int logits_dtype) {
     if (B <= 0 || K <= 0 || n <= 0 || V <= 0) return 0;
     if (logits_dtype != SPEC_BF16 && logits_dtype != SPEC_F32) return 0;
@@ -560,7 +700,7 @@ int spec_poll_error(void *workspace, void *cuda_stream) {
 }
 
 size_t spec_head_workspace_bytes(spec_handle_t h, int rows, int topk) {
-    if (!h || rows <= 0 || topk < 1 || topk > SPEC_MAX_TOPK) return 0;
+    if (!h || rows <= 0 || topk < 1 || topk > SPEC_MAX_TOPK || h->vp_ranks > 1) return 0;
     const int bn = head_block_n_for(h, rows);
     const size_t units = (size_t)rows * ((h->w.V + bn - 1) / bn);
     size_t off = kWsAlign;
@@ -572,7 +712,7 @@ size_t spec_head_workspace_bytes(spec_handle_t h, int rows, int topk) {
 }
 
 int spec_head_logits(spec_handle_t h, int level, const void *states, int rows, float *logits, void *cuda_stream) {
-    if (!h || !states || !logits || rows <= 0) return SPEC_ERR_INVALID_ARG;
+    if (!h || !states || !logits || rows <= 0 || h->vp_ranks > 1) return SPEC_ERR_INVALID_ARG;
     if (level < 0 || level >= h->w.n_heads) return SPEC_ERR_SHAPE;
     if ((uintptr_t)states & 15) return SPEC_ERR_INVALID_ARG;
     return run_gemm_store(h, states, h->w.head[level], rows, h->w.V, h->w.d_inner, head_block_n_for(h, rows), logits,
@@ -584,7 +724,7 @@ int spec_head_logits(spec_handle_t h, int level, const void *states, int rows, f
 static int head_topk_impl(spec_handle_t h, int level, const void *states, int rows, int topk, int32_t *tok, float *logp,
                           void *workspace, size_t workspace_bytes, void *cuda_stream) {
     const bool merge = tok != nullptr;
-    if (!h || !states || rows <= 0 || (merge && !logp)) return SPEC_ERR_INVALID_ARG;
+    if (!h || !states || rows <= 0 || (merge && !logp) || h->vp_ranks > 1) return SPEC_ERR_INVALID_ARG;
     if (level < 0 || level >= h->w.n_heads || topk < 1 || topk > SPEC_MAX_TOPK || topk > h->w.V) return SPEC_ERR_SHAPE;
     if ((uintptr_t)states & 15) return SPEC_ERR_INVALID_ARG;
     const size_t need = spec_head_workspace_bytes(h, rows, topk);

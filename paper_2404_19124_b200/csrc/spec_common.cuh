@@ -105,6 +105,7 @@ struct GemmEpilogue {
     int fp8;           // operands are e4m3 bytes instead of bf16; mode 1 then multiplies every accumulator by
                        // row_scale[m] * col_scale[n] before the selection
     const float *row_scale, *col_scale;
+    int idx_offset;    // mode 1: added to every column index written to part_idx (first vocabulary row of a shard)
 };
 int choose_block_n(int M, int N, int num_sm, bool tensor_bound_pref);
 int launch_gemm_tc(const void *A, const void *B, int M, int N, int Kd, int block_n, const GemmEpilogue &epi,
@@ -154,6 +155,9 @@ struct MergeArgs {
     const float *score_in;     // [rows] or null (score 0)
     int32_t *tok_out;          // [rows, topk]
     float *score_out;          // [rows, topk]
+    // Raw form (lse_out != null), for a vocabulary shard: score_out receives the logits themselves and
+    // lse_out [rows] the log-sum-exp over this shard's columns; score_in is ignored.
+    float *lse_out;
     // Last level only (seq_done != null): the CTA whose row completes a sequence's leaves prunes that
     // sequence in the same launch, so no separate prune kernel waits behind this one.
     int32_t *seq_done;         // [B] rows finished per sequence, zero before the launch
@@ -172,6 +176,12 @@ int launch_merge_rescore(const MergeArgs &g, const void *W, const void *S, int r
 int launch_draft_init(int32_t *hdr, int words, cudaStream_t st);
 int launch_mix_ln_gelu(const MixArgs &m, int rows, cudaStream_t st);
 int launch_merge_expand(const MergeArgs &g, int rows, cudaStream_t st);
+// Cross-shard merge of a vocabulary-parallel head.  Slot g (g < n_ranks, `slot_bytes` apart, starting at
+// `slots`) holds rank g's raw lists: fp32 values [rows, topk], int32 token ids [rows, topk], fp32 lse [rows].
+// Children of every row: the topk best of the n_ranks*topk entries (value desc, token id asc) with
+// score = score_in + value - log(sum_g exp(lse_g)).
+int launch_merge_shards(const void *slots, size_t slot_bytes, int n_ranks, int rows, int topk, const float *score_in,
+                        int32_t *tok_out, float *score_out, cudaStream_t st);
 int launch_prune(const float *leaf_score, const PruneArgs &pa, int B, int L, int K, int32_t *cand_tok,
                  float *cand_logp, cudaStream_t st);
 

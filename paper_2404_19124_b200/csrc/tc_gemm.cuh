@@ -490,7 +490,7 @@ __device__ __forceinline__ void epilogue_topk(const GemmJob &p, uint32_t taddr, 
                 if (!gt) --eq_left;
                 if (cnt < topk) {
                     pv[cnt] = x;
-                    pi[cnt] = col0 + c + bpos;
+                    pi[cnt] = col0 + c + bpos + p.epi.idx_offset;
                 }
                 ++cnt;
             }
