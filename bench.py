@@ -34,6 +34,9 @@ UNIT = "sequences/s"
 
 # DRAM bytes (read + write) per launch from the ncu captures summarised under profiles/ (taken with the
 # kernels as they are in this tree; set to None when a kernel changes until it is captured again)
+# Default run: about 0.6 s of timed steps at the llama2-13b shape, long enough for several clock samples.
+DEFAULT_STEPS, DEFAULT_WARMUP = 2000, 50
+
 NCU_TRAFFIC_BYTES = {
     ("llama2-13b", "head_gemm_384_rows"): 278.9e6,     # profiles/gemm_tc_kernel_head_llama2-13b.md
     ("llama2-13b", "verify_stream"): 135.2e6,          # profiles/verify_stream_kernel_llama2-13b.md
@@ -208,8 +211,8 @@ def run_only(args, cfg, peaks, dev):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=200)
-    ap.add_argument("--warmup", type=int, default=20)
+    ap.add_argument("--steps", type=int, default=DEFAULT_STEPS)
+    ap.add_argument("--warmup", type=int, default=DEFAULT_WARMUP)
     ap.add_argument("--config", default="llama2-13b")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -227,7 +230,7 @@ def main():
 
     if args.impl == "reference":
         if rank == 0:
-            if args.steps == 200 and args.warmup == 20:      # defaults are sized for the GPU arm
+            if args.steps == DEFAULT_STEPS and args.warmup == DEFAULT_WARMUP:      # defaults are sized for the GPU arm
                 args.steps, args.warmup = 3, 1
             run_reference(args, cfg)
         return
