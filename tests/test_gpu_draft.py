@@ -407,3 +407,26 @@ def test_draft_wide_states(B, d, fp8):
     cfg = small_cfg(d_base=64, d_inner=d, V=264, topk=(2, 2), K=3, B=2, seed=d % 97)
     chk = _draft_and_check(B, cfg, check_levels=not fp8, fp8=fp8)
     assert chk.exact + chk.tolerated == cfg.B
+
+
+@pytest.mark.parametrize("name,fp8", [("llama2-13b", False), ("codellama-34b", False), ("llama2-7b", True)])
+def test_draft_repeats_are_bit_identical_at_full_size(B, name, fp8):
+    """200 back-to-back drafts of the same input into rotating output buffers: the CTA that happens to finish a
+    sequence's last level also prunes it, so which CTA that is varies from run to run; the result must not."""
+    cfg = synth.CONFIGS[name]
+    sw = synth.make_weights(cfg, device="cuda")
+    h = B.spec_create(sw)
+    if fp8:
+        B.spec_attach_fp8_heads(h)
+    ctx, tok = synth.make_draft_inputs(cfg, device="cuda")
+    ws = torch.empty(B.spec_draft_workspace_bytes(h, cfg.B, cfg.topk, cfg.K), dtype=torch.uint8, device="cuda")
+    reps = 200
+    cands = torch.full((reps, cfg.B, cfg.K, cfg.n), -1, dtype=torch.int32, device="cuda")
+    logps = torch.full((reps, cfg.B, cfg.K), float("nan"), dtype=torch.float32, device="cuda")
+    for i in range(reps):
+        B.spec_draft(h, ctx, tok, cfg.topk, cfg.K, cand_tok=cands[i], cand_logp=logps[i], workspace=ws)
+    torch.cuda.synchronize()
+    assert B.spec_poll_error(ws) == 0
+    assert bool((cands == cands[0]).all()) and bool((logps == logps[0]).all())
+    assert int(cands.min()) >= 0
+    B.spec_destroy(h)
