@@ -340,6 +340,36 @@ def main():
     torch.cuda.synchronize()
     e2e_ms = max_over_ranks((time.perf_counter() - t0) * 1e3 / e2e_steps)
 
+    # ---------------------------------------------------------------- the same steps as one CUDA graph
+    # n_rot steps (one per logits buffer) captured once and replayed: what is left when the host's launch
+    # calls are taken out of the picture
+    graph_ms = None
+    try:
+        gs = torch.cuda.Stream()
+        gs.wait_stream(stream)
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.stream(gs):
+            with torch.cuda.graph(graph, stream=gs):
+                for i in range(n_rot):
+                    B.spec_draft(h, ctx, tok, cfg.topk, K, cand_tok=cand, cand_logp=logp, workspace=ws, stream=gs)
+                    B.spec_verify(cand, rot[i], accept_len=acc, best_cand=best, next_tok=nxt, workspace=vws, stream=gs)
+            replays = max(3, min(args.steps, 400) // n_rot)
+            for _ in range(3):
+                graph.replay()
+            gs.synchronize()
+            g0, g1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            g0.record(gs)
+            for _ in range(replays):
+                graph.replay()
+            g1.record(gs)
+            gs.synchronize()
+        graph_ms = max_over_ranks(g0.elapsed_time(g1) / (replays * n_rot))
+        stream.wait_stream(gs)
+        del graph
+    except RuntimeError as e:      # capture not available: the key stays null, nothing else depends on it
+        sys.stderr.write(f"graph replay skipped: {e}\n")
+    assert B.spec_poll_error(ws) == 0
+
     # ---------------------------------------------------------------- per-kernel times (CUDA events)
     B.spec_set_option(h, B.SPEC_OPT_PROFILE, 1)
     prof_steps = max(3, min(args.steps, 50))
@@ -498,6 +528,8 @@ def main():
                             "frac_of_burst": round(2.0 * bk_rows * cfg.d_inner * V / (bk_ms * 1e-3) / 1e12 / peaks["bf16_tflops"], 3)},
         "step_with_e4m3_heads": {"ms_per_step": round(fp8_step_ms, 5), "value": shard.whole_job_rate(Bn, world, fp8_step_ms * 1e-3),
                                  "what": "optional mode: e4m3 head copies on the weight-bound levels, short list re-scored in bf16"},
+        "graph_replay": {"ms_per_step": None if graph_ms is None else round(graph_ms, 5),
+                         "what": "the same draft + verify steps captured in one CUDA graph and replayed"},
         "kernel_us": kernels, "kernel_us_note": "separate-kernel form bracketed by events (adds 2-3 us per kernel); "
                                                 "the timed step launches the next level's projection with the head",
         "cpu_baseline": cpu,
