@@ -56,7 +56,9 @@ enum spec_option {
                                   the caller's stream (read them with spec_profile_read); costs a
                                   few microseconds per call, off by default                    */
     SPEC_OPT_FP8_MAX_ROWS = 4  /* levels with at most this many nodes use the e4m3 copy of their head when
-                                  one is attached (default 128; 0 = never)                     */
+                                  one is attached (default 128, the levels bound by the weight
+                                  stream; 0 = never).  Larger values put tensor-bound levels on
+                                  the e4m3 path too, which pays from about 768 nodes on        */
 };
 
 typedef struct spec_handle_s *spec_handle_t;

@@ -355,7 +355,7 @@ int spec_set_option(spec_handle_t h, int option, int value) {
             h->prof_count = 0;
             return SPEC_OK;
         case SPEC_OPT_FP8_MAX_ROWS:
-            if (value < 0 || value > 128) return SPEC_ERR_INVALID_ARG;
+            if (value < 0 || value > (1 << 24)) return SPEC_ERR_INVALID_ARG;
             h->fp8_max_rows = value;
             return SPEC_OK;
         default:

@@ -118,7 +118,7 @@ def test_head_topk_exact_ties_prefer_lower_token_id(B):
     B.spec_destroy(h)
 
 
-def _draft_and_check(B, cfg, seqs=None, impl=0, check_levels=False, tie_weights=False, fp8=False):
+def _draft_and_check(B, cfg, seqs=None, impl=0, check_levels=False, tie_weights=False, fp8=False, fp8_rows=None):
     """Runs spec_draft at the config's full batch and compares the sequences in `seqs`
     (default: all) with the oracle, one sequence at a time (sequences are independent).
     tie_weights: every head after the first aliases the second head's tensors (the weight-tied
@@ -139,6 +139,8 @@ def _draft_and_check(B, cfg, seqs=None, impl=0, check_levels=False, tie_weights=
     B.spec_set_option(h, B.SPEC_OPT_GEMM_IMPL, impl)
     if fp8:      # levels of up to 128 nodes multiply in e4m3 and re-score a short list exactly
         B.spec_attach_fp8_heads(h)
+        if fp8_rows is not None:   # also levels with more than the default 128 nodes
+            B.spec_set_option(h, B.SPEC_OPT_FP8_MAX_ROWS, fp8_rows)
     cand_tok, cand_logp, ws = B.spec_draft(h, ctx.cuda(), tok.cuda(), cfg.topk, cfg.K)
     assert B.spec_poll_error(ws) == 0
     ct, lp = cand_tok.cpu().numpy(), cand_logp.cpu().numpy()
@@ -248,6 +250,14 @@ def test_draft_fp8_heads_small_shapes(B, topk, K, Bn, V, d_base, d):
     # swap places against the oracle; every such list goes through the level-by-level check in DraftChecker
     chk = _draft_and_check(B, cfg, check_levels=False, fp8=True)
     assert chk.exact + chk.tolerated == Bn
+
+
+@pytest.mark.parametrize("topk,K,Bn", [((4, 3), 12, 60), ((2, 3, 2), 6, 90)])
+def test_draft_fp8_heads_on_levels_of_several_row_tiles(B, topk, K, Bn):
+    """SPEC_OPT_FP8_MAX_ROWS raised: levels of 240 and 540 nodes (two and five 128-row tiles) in e4m3 too."""
+    cfg = small_cfg(d_base=64, d_inner=128, V=1096, topk=topk, K=K, B=Bn, seed=Bn)
+    chk = _draft_and_check(B, cfg, seqs=range(0, Bn, 7), fp8=True, fp8_rows=4096)
+    assert chk.exact + chk.tolerated == len(range(0, Bn, 7))
 
 
 @pytest.mark.parametrize("name,seqs", [("llama2-7b", (0, 3, 7)), ("llama2-13b", (1, 9))])
