@@ -505,8 +505,10 @@ def main():
         # many sequences of the batch as fit
         probe, cores = time_oracle(cfg, sw_cpu, 1, 2)
         seqs = max(1, min(Bn, int(15.0 / min(probe))))
-        reps = max(1, min(8, int(15.0 / (min(probe) * seqs))))
+        one_pass, cores = time_oracle(cfg, sw_cpu, seqs, 1)
+        reps = max(1, min(12, int(round(15.0 / one_pass[0])) - 1))
         times, cores = time_oracle(cfg, sw_cpu, seqs, reps)
+        times = one_pass + times
         cpu = {"value": seqs * len(times) / sum(times), "unit": UNIT, "cores": cores, "kind": "oracle",
                "sample": f"{seqs} of {Bn} sequences of {cfg.name} (full draft tree + verify) x {len(times)} passes, "
                          f"{sum(times):.1f} s of oracle time"}
