@@ -23,7 +23,8 @@
  * routines (embedding, linear, layer_norm, erf-GELU, log_softmax, topk), probability
  * mass of a full tree == 1, brute-force path enumeration, the no-token-conditioning
  * special case (Sec. 3.1, the parallel-head structure), a hand-built token-conditioning
- * case, and hand-built verification examples.
+ * case, hand-built exact ties of leaf scores (all scores equal; a tie across the K
+ * boundary) for the prune's lower-leaf-first rule, and hand-built verification examples.
  * Parity unpinned: the behaviour of the authors' trained speculators (tokens per step
  * in Sec. 3.1 / Tables 1-2) - it needs their weights and data.
  */

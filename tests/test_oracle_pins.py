@@ -286,6 +286,64 @@ def test_children_depend_on_the_sampled_token():
     assert lp[0, 0] > lp[0, 1]
 
 
+def _tie_weights(V, d, n, heads, embs, d_base=4):
+    """Hand-built speculator: zero projections (the state carries nothing), identity LayerNorm affine."""
+    z = lambda *s: torch.zeros(*s)
+    bits = lambda t: synth.bf16_bits(t.to(torch.bfloat16))
+    return oracle.Weights(
+        V=V, d_base=d_base, d_inner=d, emb=[bits(t) for t in embs],
+        proj=[bits(z(d, d_base if l == 0 else d)) for l in range(n)],
+        ln_gamma=[np.ones(d, np.float32)] * n, ln_beta=[np.zeros(d, np.float32)] * n,
+        head=[bits(t) for t in heads], state_weight=1.0, emb_weight=1.0)
+
+
+@pytest.mark.parametrize("topk,K", [((3, 2, 2), 5), ((2, 2), 1), ((2, 3), 6), ((4, 4, 4, 4), 200)])
+def test_prune_with_all_scores_equal_keeps_the_lowest_leaf_indices(topk, K):
+    """All-zero output matrices: every logit is 0, so every top-k list is tokens 0..k-1 in id order with
+    log-probability -ln V each, every leaf scores -n ln V, and pruning by confidence (Sec. 4.1) with
+    equal scores must return leaves 0..K-1 in index order.  Leaf i spells i in the mixed radix topk."""
+    V, d, n = 11, 8, len(topk)
+    g = torch.Generator().manual_seed(21)
+    embs = [torch.randn(V, d, generator=g) for _ in range(n)]          # states differ per token; logits do not
+    ow = _tie_weights(V, d, n, [torch.zeros(V, d)] * n, embs)
+    ctx = synth.bf16_bits(torch.ones(2, 4, dtype=torch.bfloat16))
+    ct, lp = oracle.draft(ow, ctx, np.array([3, 7], np.int32), topk, K)
+    want = []
+    for leaf in range(K):
+        digits, rest = [], leaf
+        for k in reversed(topk):
+            digits.append(rest % k)
+            rest //= k
+        want.append(digits[::-1])
+    for b in range(2):
+        assert ct[b].tolist() == want
+    assert np.abs(lp + n * math.log(V)).max() < 1e-5
+
+
+def test_prune_tie_across_the_K_boundary_prefers_the_lower_leaf():
+    """Two head-0 tokens (5 and 9) with identical output rows and identical level-1 embeddings: their
+    subtrees score exactly alike.  Leaves in index order: 0 = (5, X), 1 = (5, Y), 2 = (9, X), 3 = (9, Y)
+    with score(0) == score(2) > score(1) == score(3); the order by (score desc, leaf asc) is 0, 2, 1, 3,
+    so K = 1 must keep leaf 0 and K = 3 must keep leaves 0, 2, 1 (Sec. 4.1 prune; ties to the lower leaf)."""
+    V, d = 12, 8
+    z = lambda *s: torch.zeros(*s)
+    emb0, emb1, head0, head1 = z(V, d), z(V, d), z(V, d), z(V, d)
+    emb0[0, 0] = 4.0                       # last_tok = 0 lights unit 0
+    head0[5, 0] = head0[9, 0] = 3.0        # ... which favours tokens 5 and 9 equally
+    emb1[5, 1] = emb1[9, 1] = 4.0          # both light unit 1 at the next stage
+    head1[2, 1], head1[7, 1] = 3.0, 2.0    # X = 2 then Y = 7
+    ow = _tie_weights(V, d, 2, [head0, head1], [emb0, emb1])
+    ctx = synth.bf16_bits(torch.ones(1, 4, dtype=torch.bfloat16))
+    tok = np.array([0], np.int32)
+    full_tok, full_lp = oracle.draft(ow, ctx, tok, (2, 2), 4)
+    assert full_tok[0].tolist() == [[5, 2], [9, 2], [5, 7], [9, 7]]
+    assert full_lp[0, 0] == full_lp[0, 1] and full_lp[0, 2] == full_lp[0, 3] and full_lp[0, 1] > full_lp[0, 2]
+    ct1, _ = oracle.draft(ow, ctx, tok, (2, 2), 1)
+    assert ct1[0].tolist() == [[5, 2]]
+    ct3, _ = oracle.draft(ow, ctx, tok, (2, 2), 3)
+    assert ct3[0].tolist() == [[5, 2], [9, 2], [5, 7]]
+
+
 # ----------------------------------------------------------------------------- verification
 def _logits_from_argmax(g, V, dtype=np.float32):
     g = np.asarray(g)
