@@ -62,6 +62,7 @@ class DraftChecker:
         self.ow, self.topk, self.K, self.n = ow, tuple(topk), K, len(topk)
         self.tolerated = 0
         self.exact = 0
+        self.max_unshared = 0     # most candidates of one tolerated sequence that the oracle's list does not hold
 
     def check(self, ctx_bits_row: np.ndarray, last_tok: int, gpu_tok: np.ndarray, gpu_logp: np.ndarray,
               levels=None, force_levels: bool = False):
@@ -82,6 +83,13 @@ class DraftChecker:
         else:
             self.tolerated += 1
             assert levels is not None, "candidate lists differ and no intermediates were given"
+            # what a near-tie can change is the order of neighbours and, at the K-th place, one membership:
+            # candidates both lists hold must carry the same score within the tolerance
+            theirs = {tuple(r): s for r, s in zip(o_tok.tolist(), o_lp.tolist())}
+            ours = {tuple(r): s for r, s in zip(gpu_tok.tolist(), gpu_logp.tolist())}
+            shared = set(theirs) & set(ours)
+            self.max_unshared = max(self.max_unshared, K - len(shared))
+            assert all(abs(theirs[c] - ours[c]) <= tol for c in shared), "shared candidates' scores differ"
         self._check_levels(ctx_bits_row, last_tok, gpu_tok, gpu_logp, levels)
 
     def _check_levels(self, ctx_bits_row, last_tok, gpu_tok, gpu_logp, lv):

@@ -291,16 +291,36 @@ def test_draft_fp8_heads_full_size(B, name, seqs):
     B.spec_destroy(h)
 
 
-def test_draft_llama2_7b_shape(B):
-    chk = _draft_and_check(B, synth.CONFIGS["llama2-7b"])
-    assert chk.tolerated <= 4      # near-ties after a bf16 rounding flip; each is checked level by level
+def _report_tolerated(record_property, name, chk, checked):
+    """The number of sequences whose candidate list differs from the oracle's at a near-tie (each of them
+    verified level by level on the GPU's own intermediates) is part of the result: print and record it."""
+    print(f"[tolerated] {name}: {chk.tolerated} of {checked} checked sequences teacher-forced, {chk.exact} exact; "
+          f"at most {chk.max_unshared} of {chk.K} candidates of such a sequence not in the oracle's list")
+    record_property("tolerated", chk.tolerated)
+    record_property("max_unshared", chk.max_unshared)
+    record_property("checked", checked)
 
 
-@pytest.mark.parametrize("name,seqs", [("llama2-13b", (0, 7, 15)), ("codellama-34b", (0, 31)), ("llama3-8b", (63,))])
-def test_draft_full_size_sampled_sequences(B, name, seqs):
+def test_draft_llama2_7b_shape(B, record_property):
+    cfg = synth.CONFIGS["llama2-7b"]
+    chk = _draft_and_check(B, cfg)
+    _report_tolerated(record_property, cfg.name, chk, cfg.B)
+    assert chk.exact + chk.tolerated == cfg.B
+    # near-ties after a bf16 rounding flip (the synthetic heads give nearly flat distributions, so leaf scores
+    # crowd together); each such sequence is checked level by level, and differs by neighbours changing places
+    assert chk.tolerated <= cfg.B // 2 and chk.max_unshared <= 2
+
+
+# one sequence of the first, a middle and the last 128-row tile of the last level at least
+@pytest.mark.parametrize("name,seqs", [("llama2-13b", (0, 3, 7, 11, 15)), ("codellama-34b", (0, 9, 15, 22, 31)),
+                                       ("llama3-8b", (0, 31, 63))])
+def test_draft_full_size_sampled_sequences(B, record_property, name, seqs):
     """Full batch on the GPU in the benchmark's launch configuration; the oracle re-computes
     whole trees for a sample of sequences (the full batch would take it minutes to hours)."""
-    _draft_and_check(B, synth.CONFIGS[name], seqs=seqs)
+    chk = _draft_and_check(B, synth.CONFIGS[name], seqs=seqs)
+    _report_tolerated(record_property, name, chk, len(seqs))
+    assert chk.exact + chk.tolerated == len(seqs)
+    assert chk.tolerated <= len(seqs) - 1 and chk.max_unshared <= 2
 
 
 def test_draft_is_deterministic_and_stream_ordered(B):
