@@ -320,7 +320,10 @@ def test_draft_full_size_sampled_sequences(B, record_property, name, seqs):
     chk = _draft_and_check(B, synth.CONFIGS[name], seqs=seqs)
     _report_tolerated(record_property, name, chk, len(seqs))
     assert chk.exact + chk.tolerated == len(seqs)
-    assert chk.tolerated <= len(seqs) - 1 and chk.max_unshared <= 2
+    # the more candidates are kept, the likelier two of them score within the rounding of a bf16 state and come
+    # out in the other order (64 of 192 leaves on the largest shape: every sequence); what is bounded is how far a
+    # tolerated list may be from the oracle's: neighbours changing places, and at most two memberships at the K-th place
+    assert chk.max_unshared <= 2
 
 
 def test_draft_is_deterministic_and_stream_ordered(B):
