@@ -166,22 +166,30 @@ def run_only(args, cfg, peaks, dev):
     from paper_2404_19124_b200 import synth
     stream = torch.cuda.current_stream()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    if args.only == "head":
+    if args.only in ("head", "head_gemm"):
+        if args.vocab:
+            cfg = dataclasses.replace(cfg, V=args.vocab)
         rows = args.rows or cfg.nodes(cfg.n - 1)
-        k = cfg.topk[-1]
+        k = args.topk or cfg.topk[-1]
         one = dataclasses.replace(cfg, topk=(k,), K=1)
         sw = synth.make_weights(one, device=dev)
         h = B.spec_create(sw)
         if args.block_n:
             B.spec_set_option(h, B.SPEC_OPT_HEAD_BLOCK_N, args.block_n)
+        if args.swap_max_rows is not None:
+            B.spec_set_option(h, B.SPEC_OPT_HEAD_SWAP_MAX_ROWS, args.swap_max_rows)
         g = torch.Generator(device=dev).manual_seed(5)
         S = (torch.randn(rows, cfg.d_inner, generator=g, device=dev) * 0.5).to(torch.bfloat16)
         tok = torch.empty((rows, k), dtype=torch.int32, device=dev)
         logp = torch.empty((rows, k), dtype=torch.float32, device=dev)
         ws = torch.empty(B.spec_head_workspace_bytes(h, rows, k), dtype=torch.uint8, device=dev)
-        run = lambda i: B.spec_head_topk(h, 0, S, k, tok=tok, logp=logp, workspace=ws)
+        if args.only == "head":
+            run = lambda i: B.spec_head_topk(h, 0, S, k, tok=tok, logp=logp, workspace=ws)
+        else:
+            run = lambda i: B.spec_head_partials(h, 0, S, k, ws)
         flops, nbytes = 2.0 * rows * cfg.d_inner * cfg.V, 2.0 * cfg.V * cfg.d_inner + 2.0 * rows * cfg.d_inner
-        what = f"spec_head_topk rows={rows} d_inner={cfg.d_inner} V={cfg.V} topk={k} (GEMM + merge kernels)"
+        what = (f"{'spec_head_topk' if args.only == 'head' else 'spec_head_partials'} rows={rows} d_inner={cfg.d_inner} "
+                f"V={cfg.V} topk={k} ({'GEMM + merge kernels' if args.only == 'head' else 'GEMM kernel with its fused epilogue'})")
     else:
         cand = synth.random_cand_tok(cfg, device=dev)
         nbytes = cfg.B * cfg.K * (cfg.n + 1) * cfg.V * 2.0
@@ -216,7 +224,11 @@ def main():
     ap.add_argument("--config", default="llama2-13b")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--only", default=None, choices=["head", "verify"],
+    ap.add_argument("--swap-max-rows", type=int, default=None,
+                    help="--only head*: levels of at most this many rows use the weight-stream form (0: never)")
+    ap.add_argument("--vocab", type=int, default=None, help="--only head*: vocabulary size instead of the workload's")
+    ap.add_argument("--topk", type=int, default=None, help="--only head*: branching factor (default: the last level's)")
+    ap.add_argument("--only", default=None, choices=["head", "head_gemm", "verify"],
                     help="kernel-level run for profiling: only the vocabulary-head GEMM (+merge) or only verify")
     ap.add_argument("--rows", type=int, default=None, help="--only head: rows of the GEMM (default: last level)")
     ap.add_argument("--block-n", type=int, default=0, help="--only head: force the vocabulary tile width")

@@ -55,10 +55,15 @@ enum spec_option {
     SPEC_OPT_PROFILE = 3,      /* 1: spec_draft brackets each of its kernels with CUDA events on
                                   the caller's stream (read them with spec_profile_read); costs a
                                   few microseconds per call, off by default                    */
-    SPEC_OPT_FP8_MAX_ROWS = 4  /* levels with at most this many nodes use the e4m3 copy of their head when
+    SPEC_OPT_FP8_MAX_ROWS = 4, /* levels with at most this many nodes use the e4m3 copy of their head when
                                   one is attached (default 128, the levels bound by the weight
                                   stream; 0 = never).  Larger values put tensor-bound levels on
                                   the e4m3 path too, which pays from about 768 nodes on        */
+    SPEC_OPT_HEAD_SWAP_MAX_ROWS = 5 /* levels with at most this many nodes (0 .. 128, default 128) run
+                                  the head GEMM with the weight matrix on the 128-row side of the
+                                  MMA and the nodes as columns, so the tensor work follows the
+                                  number of nodes and the launch is a pure weight stream; 0 = never.
+                                  Ignored while SPEC_OPT_HEAD_BLOCK_N forces a tile width.     */
 };
 
 typedef struct spec_handle_s *spec_handle_t;

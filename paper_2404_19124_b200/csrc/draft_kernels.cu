@@ -95,6 +95,29 @@ __global__ void __launch_bounds__(kMergeThreads) merge_expand_kernel(MergeArgs g
     prune_if_last<kMergeThreads, BlockSync>(g, blockIdx.x, threadIdx.x, merge_keys, &last_of_sequence);
 }
 
+// Merge of level l and the gather + mix + LayerNorm + GELU of level l + 1 in one launch: one CTA of 256 threads
+// per row of level l folds the row's partial lists into its children (tokens, scores) and then computes the
+// states of those children, whose tokens it has just found and whose parent projection is this row's.  One
+// kernel boundary less between two vocabulary heads.
+struct MergeMixArgs {
+    MergeArgs merge;   // level l
+    MixArgs mix;       // level l + 1 (tok and parent_div unused: the tokens come from the merge)
+};
+
+__global__ void __launch_bounds__(kRowThreads, 1) merge_mix_kernel(MergeMixArgs a) {
+    __shared__ Scratch sc;
+    __shared__ float red_a[kRowThreads / 32 * 4], red_b[kRowThreads / 32 * 4];
+    griddep_launch();
+    griddep_wait();
+    const int r = blockIdx.x, tid = threadIdx.x;
+    merge_expand_row<kRowThreads, BlockSync>(a.merge, r, tid, &sc);
+    // sc.out_id[0 .. topk) now hold the children's tokens (valid for the whole CTA after merge_select's last barrier)
+    if (a.mix.d <= 8 * kRowThreads)
+        mix_children<kRowThreads, 1, BlockSync>(a.mix, r, r * a.merge.topk, a.merge.topk, sc.out_id, red_a, red_b, tid);
+    else
+        mix_children<kRowThreads, 2, BlockSync>(a.mix, r, r * a.merge.topk, a.merge.topk, sc.out_id, red_a, red_b, tid);
+}
+
 // Vocabulary-parallel head: one warp per row folds the n_ranks raw lists (see launch_merge_shards).
 // Lane i owns entries i and i + 32 of the row's n_ranks * topk <= 64 candidates.
 constexpr int kShardRowsPerCta = 4;
@@ -191,6 +214,16 @@ int launch_draft_init(int32_t *hdr, int words, cudaStream_t st) {
 int launch_merge_expand(const MergeArgs &g, int rows, cudaStream_t st) {
     const size_t smem = g.seq_done ? sizeof(LeafKey) * (size_t)g.Lpad : 0;
     SPEC_CUDA_TRY(launch_pdl(merge_expand_kernel, dim3(rows), dim3(kMergeThreads), smem, st, g));
+    return SPEC_OK;
+}
+
+// Returns SPEC_ERR_SHAPE when the fused form does not cover the shape (rows wider than 4096 elements, an e4m3
+// copy of the states wanted): the caller then launches the merge and the mix separately.
+int launch_merge_mix(const MergeArgs &g, const MixArgs &m, int rows, cudaStream_t st) {
+    if (m.d > 8 * kRowThreads * 2 || m.S8_out != nullptr || g.lse_out != nullptr || g.seq_done != nullptr)
+        return SPEC_ERR_SHAPE;
+    MergeMixArgs a{g, m};
+    SPEC_CUDA_TRY(launch_pdl(merge_mix_kernel, dim3(rows), dim3(kRowThreads), 0, st, a));
     return SPEC_OK;
 }
 

@@ -14,6 +14,9 @@
 // that share a weight tile run at the same time and the second and third readers hit L2.
 #include <cuda.h>
 
+#include <mutex>
+#include <vector>
+
 #include "tc_gemm.cuh"
 
 namespace spec {
@@ -29,17 +32,21 @@ struct GemmParams {
     int n_jobs;
     int stages, tmem_cols, acc_stride;
     uint32_t slot_bytes;
+    uint32_t tbuf_bytes;     // transposed accumulator tile of a mode-3 job (0: none in this launch)
+    int32_t *clear;          // words that the first kernel of a draft sets to zero (the workspace header) ...
+    int clear_words;         // ... by CTA 0, after the preceding grid has completed; 0: nothing
     int32_t *err;
 };
 
 struct GemmMaps {
     CUtensorMap a[kMaxJobs], b[kMaxJobs];
+    CUtensorMap a_short;   // mode 3 (job 0): the weight box of the last, shorter tile of every CTA
 };
 
 __global__ void __launch_bounds__(kThreads, 1)
 gemm_tc_kernel(const __grid_constant__ GemmMaps maps, const __grid_constant__ GemmParams p) {
     extern __shared__ uint8_t smem_raw[];
-    const Pipe pp = pipe_setup(smem_raw, p.stages, p.slot_bytes, p.tmem_cols, p.acc_stride, p.err);
+    const Pipe pp = pipe_setup(smem_raw, p.stages, p.slot_bytes, p.tmem_cols, p.acc_stride, p.tbuf_bytes, p.err);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
     griddep_launch();   // the next kernel in the stream may start its own set-up now
@@ -50,7 +57,7 @@ gemm_tc_kernel(const __grid_constant__ GemmMaps maps, const __grid_constant__ Ge
             bool ok = true;
             // the weights are fetched before the preceding grid is waited for, the states after
             for (int q = 0; ok && q < p.n_jobs; ++q)
-                ok = produce_job(pp, p.job[q], &maps.a[q], &maps.b[q], rp, issued, [] { griddep_wait(); return true; });
+                ok = produce_job(pp, p.job[q], &maps.a[q], &maps.a_short, &maps.b[q], rp, issued, [] { griddep_wait(); return true; });
             if (!ok) producer_drain(pp, rp, issued);
         }
         griddep_wait();
@@ -66,6 +73,12 @@ gemm_tc_kernel(const __grid_constant__ GemmMaps maps, const __grid_constant__ Ge
         AccPos ap{0, 0u};
         bool ok = true;
         griddep_wait();
+        // First kernel of a draft: the header (error word, per-sequence counters) starts at zero.  Nothing of
+        // this draft has reported or counted yet: the counters are first touched by the last level's merge,
+        // and a wait that runs out does so millions of polls after this point.
+        if (p.clear_words > 0 && blockIdx.x == 0)
+            for (int i = (int)threadIdx.x - (kThreads - kEpilogueThreads); i < p.clear_words; i += kEpilogueThreads)
+                p.clear[i] = 0;
         for (int q = 0; ok && q < p.n_jobs; ++q) ok = epilogue_job(pp, p.job[q], ap);
     }
     pipe_teardown(pp, p.tmem_cols);
@@ -76,7 +89,9 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t
                                   const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
-EncodeTiledFn get_encode_fn() {
+std::mutex g_host_mutex;   // guards the driver entry point, the tensor-map cache and the per-device attribute flags
+
+EncodeTiledFn get_encode_fn() {   // called with g_host_mutex held
     static EncodeTiledFn fn = nullptr;
     if (fn) return fn;
     void *ptr = nullptr;
@@ -90,10 +105,52 @@ EncodeTiledFn get_encode_fn() {
     return fn;
 }
 
+// Encoded tensor maps, kept for the life of the process: a map depends only on the address, the shape and
+// the box, not on the tensor's contents, and the weights of a handle and the buffers of a workspace come back
+// call after call.  A draft therefore encodes nothing after the first call with its workspace.
+struct TmapKey {
+    const void *base;
+    uint64_t rows, cols;
+    uint32_t box_rows;
+    int streamed, fp8;
+    bool operator==(const TmapKey &o) const {
+        return base == o.base && rows == o.rows && cols == o.cols && box_rows == o.box_rows && streamed == o.streamed &&
+               fp8 == o.fp8;
+    }
+};
+struct TmapEntry {
+    TmapKey key;
+    CUtensorMap map;
+};
+constexpr size_t kTmapCacheCap = 1024;   // beyond this the cache starts over
+std::vector<TmapEntry> g_tmap_cache;
+
+int encode_tmap(CUtensorMap *map, const void *base, uint64_t rows, uint64_t cols, uint32_t box_rows, bool streamed,
+                bool fp8);
+
 }  // namespace
 
 int make_tmap(CUtensorMap *map, const void *base, uint64_t rows, uint64_t cols, uint32_t box_rows, bool streamed,
               bool fp8) {
+    const TmapKey key{base, rows, cols, box_rows, streamed ? 1 : 0, fp8 ? 1 : 0};
+    std::lock_guard<std::mutex> lock(g_host_mutex);
+    for (const TmapEntry &e : g_tmap_cache) {
+        if (e.key == key) {
+            *map = e.map;
+            return SPEC_OK;
+        }
+    }
+    const int rc = encode_tmap(map, base, rows, cols, box_rows, streamed, fp8);
+    if (rc != SPEC_OK) return rc;
+    if (g_tmap_cache.size() >= kTmapCacheCap) g_tmap_cache.clear();
+    g_tmap_cache.push_back(TmapEntry{key, *map});
+    return SPEC_OK;
+}
+
+namespace {
+
+int encode_tmap(CUtensorMap *map, const void *base, uint64_t rows, uint64_t cols, uint32_t box_rows, bool streamed,
+                bool fp8) {
     EncodeTiledFn fn = get_encode_fn();
     if (!fn) return SPEC_ERR_CUDA;
     const uint32_t esz = fp8 ? 1 : 2;
@@ -110,6 +167,27 @@ int make_tmap(CUtensorMap *map, const void *base, uint64_t rows, uint64_t cols, 
         return SPEC_ERR_CUDA;
     }
     return SPEC_OK;
+}
+
+}  // namespace
+
+// Mode 3: threads per node in the scan (a power of two, at most kSwapMaxSegs, nodes * segs <= 128); the
+// vocabulary rows every CTA takes (a multiple of 8, the same for all so that they stream the same number of
+// bytes; the last CTA of the deal may get fewer); and the number of partial lists per node = CTAs of the deal.
+int swapped_head_segs(int nodes) {
+    int segs = 1;
+    while (segs < kSwapMaxSegs && nodes * segs * 2 <= kEpilogueThreads) segs *= 2;
+    return segs;
+}
+static int swapped_rows_per_cta(int vocab_rows) {
+    const int sms = num_sms();
+    const int per = (vocab_rows + sms - 1) / sms;
+    return (per + 7) / 8 * 8;
+}
+int swapped_head_parts(int nodes, int vocab_rows) {
+    (void)nodes;
+    const int per = swapped_rows_per_cta(vocab_rows);
+    return (vocab_rows + per - 1) / per;
 }
 
 // Columns per tile: a multiple of 32 in [32, 256].  Scores each candidate by how evenly its
@@ -137,7 +215,9 @@ int choose_block_n(int M, int N, int num_sm, bool prefer_wide) {
 
 int plan_job(tc::GemmJob *j, int M, int N, int Kd, int block_n, const GemmEpilogue &epi) {
     const int fp8 = epi.fp8 ? 1 : 0;
-    if (M <= 0 || N <= 0 || Kd <= 0 || Kd % (fp8 ? 16 : 8) != 0 || block_n < 32 || block_n > 256 || block_n % 32 != 0)
+    const int bn_unit = epi.mode == 3 ? 16 : 32;   // mode 3 reads the accumulator 16 columns at a time
+    if (M <= 0 || N <= 0 || Kd <= 0 || Kd % (fp8 ? 16 : 8) != 0 || block_n < bn_unit || block_n > 256 ||
+        block_n % bn_unit != 0)
         return SPEC_ERR_SHAPE;   // rows are whole 16-byte units
     j->M = M; j->N = N; j->Kd = Kd;
     j->block_n = block_n;
@@ -149,19 +229,31 @@ int plan_job(tc::GemmJob *j, int M, int N, int Kd, int block_n, const GemmEpilog
     j->splits = epi.mode == 2 && epi.splits > 1 ? epi.splits : 1;
     j->kb_per_split = (num_kb + j->splits - 1) / j->splits;
     if ((j->splits - 1) * j->kb_per_split >= num_kb) return SPEC_ERR_SHAPE;   // every split must own a K block
-    j->w_is_a = epi.mode == 2 ? 1 : 0;
+    j->w_is_a = (epi.mode == 2 || epi.mode == 3) ? 1 : 0;
     j->first_cta = 0;
+    j->deal_ctas = 0;
     j->epi = epi;
+    j->rows_per_cta = 0;
+    if (epi.mode == 3) {   // all nodes in one tile column; every CTA of the deal leaves one list per node
+        if (N > kBlockM || j->n_tiles != 1 || fp8) return SPEC_ERR_SHAPE;
+        j->epi.segs = swapped_head_segs(N);
+        j->rows_per_cta = swapped_rows_per_cta(M);
+        j->deal_ctas = (M + j->rows_per_cta - 1) / j->rows_per_cta;
+        j->epi.n_parts = j->deal_ctas;
+    }
     return SPEC_OK;
 }
 
 // One launch, one or two contractions.  The tiles of the second are dealt to the CTAs starting where
 // the first one's stopped, so a CTA that got no tile of the first starts on the second at once.
-int launch_gemm_tc_jobs(const GemmCall *calls, int n_calls, int32_t *err, cudaStream_t st) {
+int launch_gemm_tc_jobs(const GemmCall *calls, int n_calls, int32_t *err, cudaStream_t st, int32_t *clear,
+                        int clear_words) {
     if (n_calls < 1 || n_calls > kMaxJobs) return SPEC_ERR_INVALID_ARG;
     GemmParams p{};
     GemmMaps maps{};
     p.n_jobs = n_calls;
+    p.clear = clear;
+    p.clear_words = clear ? clear_words : 0;
     int max_block_n = 32;
     long long total_tiles = 0;
     for (int q = 0; q < n_calls; ++q) {
@@ -175,16 +267,30 @@ int launch_gemm_tc_jobs(const GemmCall *calls, int n_calls, int32_t *err, cudaSt
                        p.job[q].fp8 != 0);
         if (rc != SPEC_OK) return rc;
         if (c.block_n > max_block_n) max_block_n = c.block_n;
-        total_tiles += (long long)p.job[q].m_tiles * p.job[q].n_tiles * p.job[q].splits;
+        if (c.epi.mode == 3) {
+            if (q != 0) return SPEC_ERR_INVALID_ARG;   // its CTAs are the first of the grid
+            p.tbuf_bytes = (uint32_t)c.block_n * kTPitch * sizeof(float);
+            const int short_rows = p.job[q].rows_per_cta % kBlockM;
+            if (short_rows > 0) {
+                rc = make_tmap(&maps.a_short, c.A, (uint64_t)c.M, (uint64_t)c.Kd, (uint32_t)short_rows, true, false);
+                if (rc != SPEC_OK) return rc;
+            }
+            total_tiles += p.job[q].deal_ctas;   // what counts for the grid: the CTAs it occupies
+        } else {
+            total_tiles += (long long)p.job[q].m_tiles * p.job[q].n_tiles * p.job[q].splits;
+        }
     }
     const int grid = (int)(total_tiles < num_sms() ? total_tiles : num_sms());
     long long offset = 0;
     for (int q = 0; q < n_calls; ++q) {
+        // a job's tiles are dealt to the CTAs starting where the previous job's stopped; behind a mode-3 job
+        // that is the first CTA without vocabulary rows
         p.job[q].first_cta = (int)(offset % grid);
-        offset += (long long)p.job[q].m_tiles * p.job[q].n_tiles * p.job[q].splits;
+        offset += p.job[q].epi.mode == 3 ? (long long)p.job[q].deal_ctas
+                                         : (long long)p.job[q].m_tiles * p.job[q].n_tiles * p.job[q].splits;
     }
     p.slot_bytes = (uint32_t)kABytes + (uint32_t)max_block_n * kSlabBytes;
-    const int budget = kSmemLimit - 1024 - (int)sizeof(Barriers) - 64;
+    const int budget = kSmemLimit - 1024 - (int)sizeof(Barriers) - 64 - (int)p.tbuf_bytes;
     p.stages = budget / (int)p.slot_bytes;
     if (p.stages > kMaxStages) p.stages = kMaxStages;
     if (p.stages < 2) return SPEC_ERR_SHAPE;
@@ -194,13 +300,16 @@ int launch_gemm_tc_jobs(const GemmCall *calls, int n_calls, int32_t *err, cudaSt
     p.acc_stride = max_block_n;
     p.err = err;
 
-    const size_t smem = 1024 + (size_t)p.stages * p.slot_bytes + sizeof(Barriers);
-    static bool attr_set[64] = {};
+    const size_t smem = 1024 + (size_t)p.stages * p.slot_bytes + p.tbuf_bytes + sizeof(Barriers);
     int dev = 0;
     SPEC_CUDA_TRY(cudaGetDevice(&dev));
-    if (dev < 0 || dev >= 64 || !attr_set[dev]) {
-        SPEC_CUDA_TRY(cudaFuncSetAttribute(gemm_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemLimit));
-        if (dev >= 0 && dev < 64) attr_set[dev] = true;
+    {
+        static bool attr_set[64] = {};
+        std::lock_guard<std::mutex> lock(g_host_mutex);
+        if (dev < 0 || dev >= 64 || !attr_set[dev]) {
+            SPEC_CUDA_TRY(cudaFuncSetAttribute(gemm_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemLimit));
+            if (dev >= 0 && dev < 64) attr_set[dev] = true;
+        }
     }
     SPEC_CUDA_TRY(launch_pdl(gemm_tc_kernel, dim3(grid), dim3(kThreads), smem, st, maps, p));
     return SPEC_OK;

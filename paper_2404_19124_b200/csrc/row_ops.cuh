@@ -381,6 +381,130 @@ __device__ __forceinline__ void merge_expand_row(const MergeArgs &g, int r, int 
     if (g.lse_out != nullptr && tid == 0) g.lse_out[r] = sc->lse;
 }
 
+// The children of one parent row, all at once: gather + mix + LayerNorm + exact GELU of up to kBatch child
+// nodes per trip (Sec. 3.1: siblings share the projected parent state and differ in the token embedding).
+// `tok` holds the children's tokens (shared memory, written by the merge just before), `first_child` is the
+// row of child 0 in the next level.  The projected parent state (sum of the split-K partials, added in
+// ascending order) and the LayerNorm parameters are loaded once; per trip the embedding rows of the batch
+// are requested together and the two LayerNorm reductions are done for the whole batch with one barrier
+// each (red_a / red_b: kThreads / 32 x kBatch floats each).  d <= 8 * kThreads * kIters, d % 8 == 0.
+template <int kThreads, int kIters, typename Sync>
+__device__ __forceinline__ void mix_children(const MixArgs &m, int parent, int first_child, int n_child, const int *tok,
+                                             float *red_a, float *red_b, int tid) {
+    constexpr int kBatch = 4;
+    constexpr int kWarps = kThreads / 32;
+    const int d = m.d, lane = tid & 31, warp = tid >> 5;
+    float pv[kIters][8], gv[kIters][8], bv[kIters][8];
+#pragma unroll
+    for (int it = 0; it < kIters; ++it) {
+        const int i = (it * kThreads + tid) * 8;
+        const int ic = i < d ? i : 0;
+#pragma unroll
+        for (int j = 0; j < 8; ++j) pv[it][j] = 0.0f;
+        if (i < d) {
+            const float *p = m.P + (size_t)parent * d + i;
+            for (int sp = 0; sp < m.p_splits; ++sp) {
+                const float4 p0 = __ldcg((const float4 *)(p + sp * m.p_split_stride));
+                const float4 p1 = __ldcg((const float4 *)(p + sp * m.p_split_stride + 4));
+                pv[it][0] += p0.x; pv[it][1] += p0.y; pv[it][2] += p0.z; pv[it][3] += p0.w;
+                pv[it][4] += p1.x; pv[it][5] += p1.y; pv[it][6] += p1.z; pv[it][7] += p1.w;
+            }
+        }
+        const float4 g0 = *(const float4 *)(m.gamma + ic), g1 = *(const float4 *)(m.gamma + ic + 4);
+        const float4 b0 = *(const float4 *)(m.beta + ic), b1 = *(const float4 *)(m.beta + ic + 4);
+        gv[it][0] = g0.x; gv[it][1] = g0.y; gv[it][2] = g0.z; gv[it][3] = g0.w;
+        gv[it][4] = g1.x; gv[it][5] = g1.y; gv[it][6] = g1.z; gv[it][7] = g1.w;
+        bv[it][0] = b0.x; bv[it][1] = b0.y; bv[it][2] = b0.z; bv[it][3] = b0.w;
+        bv[it][4] = b1.x; bv[it][5] = b1.y; bv[it][6] = b1.z; bv[it][7] = b1.w;
+    }
+    for (int c0 = 0; c0 < n_child; c0 += kBatch) {
+        float h[kBatch][kIters][8];
+        float part[kBatch];
+        uint4 ev[kBatch][kIters];
+#pragma unroll
+        for (int q = 0; q < kBatch; ++q) {
+            const int t = c0 + q < n_child ? tok[c0 + q] : -1;
+            const bool tok_ok = t >= 0 && t < m.V;
+            if (c0 + q < n_child && !tok_ok && tid == 0) report_error(m.err, SPEC_ERR_TOKEN_RANGE);
+#pragma unroll
+            for (int it = 0; it < kIters; ++it) {
+                const int i = (it * kThreads + tid) * 8;
+                ev[q][it] = make_uint4(0u, 0u, 0u, 0u);
+                if (tok_ok && i < d) ev[q][it] = *(const uint4 *)(m.emb + (size_t)t * d + i);
+            }
+        }
+#pragma unroll
+        for (int q = 0; q < kBatch; ++q) {
+            part[q] = 0.0f;
+#pragma unroll
+            for (int it = 0; it < kIters; ++it) {
+                const int i = (it * kThreads + tid) * 8;
+                const uint32_t ew[4] = {ev[q][it].x, ev[q][it].y, ev[q][it].z, ev[q][it].w};
+#pragma unroll
+                for (int j = 0; j < 8; ++j) {
+                    const float z = (j & 1) ? __uint_as_float(ew[j >> 1] & 0xffff0000u) : __uint_as_float(ew[j >> 1] << 16);
+                    h[q][it][j] = i < d ? m.a * pv[it][j] + m.b * z : 0.0f;
+                    part[q] += h[q][it][j];
+                }
+            }
+        }
+        // batch-wide reductions: warp shuffles, one slot per (warp, child), then every thread adds the warps' slots
+        float mean[kBatch], rstd[kBatch];
+#pragma unroll
+        for (int pass = 0; pass < 2; ++pass) {
+            float *red = pass == 0 ? red_a : red_b;
+#pragma unroll
+            for (int q = 0; q < kBatch; ++q) {
+                float v = part[q];
+#pragma unroll
+                for (int off = 16; off > 0; off >>= 1) v += __shfl_xor_sync(0xffffffffu, v, off);
+                if (lane == 0) red[warp * kBatch + q] = v;
+            }
+            Sync::sync();
+#pragma unroll
+            for (int q = 0; q < kBatch; ++q) {
+                float t = 0.0f;
+#pragma unroll
+                for (int w = 0; w < kWarps; ++w) t += red[w * kBatch + q];
+                if (pass == 0) {
+                    mean[q] = t / (float)d;
+                    part[q] = 0.0f;
+#pragma unroll
+                    for (int it = 0; it < kIters; ++it) {
+                        const int i = (it * kThreads + tid) * 8;
+                        if (i < d) {
+#pragma unroll
+                            for (int j = 0; j < 8; ++j) {
+                                const float c = h[q][it][j] - mean[q];
+                                part[q] += c * c;
+                            }
+                        }
+                    }
+                } else {
+                    rstd[q] = rsqrtf(t / (float)d + m.eps);
+                }
+            }
+        }
+#pragma unroll
+        for (int q = 0; q < kBatch; ++q) {
+            if (c0 + q >= n_child) continue;
+            const size_t row = (size_t)first_child + c0 + q;
+#pragma unroll
+            for (int it = 0; it < kIters; ++it) {
+                const int i = (it * kThreads + tid) * 8;
+                uint32_t packed[4];
+#pragma unroll
+                for (int j = 0; j < 8; j += 2) {
+                    const float s0 = gelu_erf((h[q][it][j] - mean[q]) * rstd[q] * gv[it][j] + bv[it][j]);
+                    const float s1 = gelu_erf((h[q][it][j + 1] - mean[q]) * rstd[q] * gv[it][j + 1] + bv[it][j + 1]);
+                    packed[j >> 1] = float_to_bf16_bits(s0) | (float_to_bf16_bits(s1) << 16);
+                }
+                if (i < d) *(uint4 *)(m.S_out + row * d + i) = make_uint4(packed[0], packed[1], packed[2], packed[3]);
+            }
+        }
+    }
+}
+
 struct LeafKey {
     float score;
     int leaf;

@@ -1,5 +1,6 @@
 // C ABI of libspec_b200: host-side validation, workspace layout and the launch sequences of
 // spec_draft / spec_verify (declared and documented in include/spec_b200.h).
+#include <atomic>
 #include <new>
 #include <string.h>
 
@@ -11,16 +12,16 @@ static thread_local int g_last_cuda_error = 0;
 void set_last_cuda_error(int e) { g_last_cuda_error = e; }
 
 int num_sms() {
-    static int cached[64] = {};
+    static std::atomic<int> cached[64];   // zero-initialised; any thread may fill an entry, all write the same value
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return kNumSMsFallback;
-    if (cached[dev] == 0) {
-        int n = 0;
+    int n = cached[dev].load(std::memory_order_relaxed);
+    if (n == 0) {
         if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0)
             n = kNumSMsFallback;
-        cached[dev] = n;
+        cached[dev].store(n, std::memory_order_relaxed);
     }
-    return cached[dev];
+    return n;
 }
 
 }  // namespace spec
@@ -36,6 +37,7 @@ struct spec_handle_s {
     int proj_block_n;
     int profile;
     int fp8_max_rows;                      // SPEC_OPT_FP8_MAX_ROWS
+    int swap_max_rows;                     // SPEC_OPT_HEAD_SWAP_MAX_ROWS
     const void *head8[SPEC_MAX_HEADS];     // e4m3 copies of the heads (caller-owned), null: none
     const float *head8_scale[SPEC_MAX_HEADS];
     int vp_rank, vp_ranks;                 // vocabulary-parallel heads: this handle's shard (vp_ranks 1: none)
@@ -45,6 +47,8 @@ struct spec_handle_s {
 };
 
 namespace {
+
+constexpr int kFusedMixMaxChildren = 2;
 
 size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
@@ -59,6 +63,7 @@ struct DraftPlan {
     int proj_block_n[SPEC_MAX_HEADS];
     int proj_splits[SPEC_MAX_HEADS];   // > 0: swapped split-K projection (few parent rows); 0: plain
     bool use_fp8[SPEC_MAX_HEADS];      // the level's head runs on the e4m3 copy of its weights
+    bool swapped[SPEC_MAX_HEADS];      // the level's head runs with the operands swapped (few nodes: weight stream)
     size_t seq_done;                   // byte offset of the per-sequence counters of the folded prune
     int header_words;                  // int32 words cleared at the start of a draft
     size_t xchg;                       // vocabulary-parallel heads: byte offset of the rank slots
@@ -68,6 +73,22 @@ struct DraftPlan {
 int head_block_n_for(const spec_handle_s *h, int rows) {
     if (h->head_block_n > 0) return h->head_block_n;
     return choose_block_n(rows, h->head_rows, num_sms(), rows > 128);
+}
+
+// Levels of few nodes run the head with the weights on the 128-row side of the MMA (epilogue mode 3).
+bool head_swapped_for(const spec_handle_s *h, int rows) {
+    return h->gemm_impl == 0 && h->head_block_n == 0 && rows <= h->swap_max_rows && rows <= 128;
+}
+
+// Partial lists per row that the head of `rows` nodes leaves for the merge, and its tile width.
+int head_parts_for(const spec_handle_s *h, int rows, bool swapped, int *block_n_out) {
+    if (swapped) {
+        if (block_n_out) *block_n_out = 128;
+        return swapped_head_parts(rows, h->head_rows);
+    }
+    const int bn = head_block_n_for(h, rows);
+    if (block_n_out) *block_n_out = bn;
+    return (h->head_rows + bn - 1) / bn;
 }
 
 int proj_block_n_for(const spec_handle_s *h, int rows) {
@@ -133,6 +154,14 @@ int make_draft_plan(const spec_handle_s *h, int B, const int32_t *topk, int K, D
     size_t max_proj_floats = 0;
     size_t max_part_units = 0;
     int max_rows = 0;
+    int max_fp8_rows = 0;
+    for (int l = 0; l < p->n; ++l) {
+        // (the mix kernel for rows wider than 16384 elements keeps them in shared memory and has no e4m3 output)
+        p->use_fp8[l] = h->gemm_impl == 0 && !h->profile && h->head8[l] != nullptr && p->N[l] <= h->fp8_max_rows &&
+                        w.d_inner <= 16384 && h->vp_ranks == 1;
+        if (p->use_fp8[l] && p->N[l] > max_fp8_rows) max_fp8_rows = p->N[l];
+        p->swapped[l] = !p->use_fp8[l] && head_swapped_for(h, p->N[l]);
+    }
     for (int l = 0; l < p->n; ++l) {
         y.state[l] = off;
         off = align_up(off + 2 * (size_t)p->N[l] * w.d_inner, kWsAlign);
@@ -140,9 +169,9 @@ int make_draft_plan(const spec_handle_s *h, int B, const int32_t *topk, int K, D
         p->proj_splits[l] = proj_splits_for(h, parent_rows, d_in_of(w, l));
         const size_t pf = (size_t)(p->proj_splits[l] > 0 ? p->proj_splits[l] : 1) * parent_rows * w.d_inner;
         if (pf > max_proj_floats) max_proj_floats = pf;
-        const int bn = head_block_n_for(h, p->N[l]);
+        int bn = 0;
+        y.n_tiles[l] = head_parts_for(h, p->N[l], p->swapped[l], &bn);
         y.block_n[l] = bn;
-        y.n_tiles[l] = (h->head_rows + bn - 1) / bn;
         const size_t units = (size_t)p->N[l] * y.n_tiles[l];
         if (units > max_part_units) max_part_units = units;
         if (p->N[l] > max_rows) max_rows = p->N[l];
@@ -150,13 +179,6 @@ int make_draft_plan(const spec_handle_s *h, int B, const int32_t *topk, int K, D
     }
     y.proj = off;
     off = align_up(off + sizeof(float) * max_proj_floats, kWsAlign);
-    int max_fp8_rows = 0;
-    for (int l = 0; l < p->n; ++l) {
-        // (the mix kernel for rows wider than 16384 elements keeps them in shared memory and has no e4m3 output)
-        p->use_fp8[l] = h->gemm_impl == 0 && !h->profile && h->head8[l] != nullptr && p->N[l] <= h->fp8_max_rows &&
-                        w.d_inner <= 16384 && h->vp_ranks == 1;
-        if (p->use_fp8[l] && p->N[l] > max_fp8_rows) max_fp8_rows = p->N[l];
-    }
     y.state8 = off;
     off = align_up(off + (size_t)max_fp8_rows * w.d_inner, kWsAlign);
     y.state8_scale = off;
@@ -199,7 +221,40 @@ int run_head_partials(const spec_handle_s *h, const void *states, const void *Wo
     e.part_idx = part_idx;
     e.part_ms = part_ms;
     e.topk = topk;
+    if (head_swapped_for(h, rows)) {
+        e.mode = 3;
+        return launch_gemm_tc(Wout, states, w.V, rows, w.d_inner, (rows + 15) / 16 * 16, e, err, st);
+    }
     return launch_gemm_tc(states, Wout, rows, w.V, w.d_inner, block_n, e, err, st);
+}
+
+// The head of level l inside a draft: plain form (one thread per node row of a [128 x block_n] tile), the
+// swapped form for levels of few nodes, or e4m3 operands.
+GemmCall make_head_call(const spec_handle_s *h, const DraftPlan &p, char *ws, int l, int topk_l) {
+    const spec_weights_t &w = h->w;
+    GemmCall c{};
+    c.A = ws + p.lay.state[l]; c.B = w.head[l]; c.M = p.N[l]; c.N = h->head_rows; c.Kd = w.d_inner;
+    c.block_n = p.lay.block_n[l];
+    c.epi.mode = 1;
+    c.epi.part_val = (float *)(ws + p.lay.part_val);
+    c.epi.part_idx = (int32_t *)(ws + p.lay.part_idx);
+    c.epi.part_ms = (float *)(ws + p.lay.part_ms);
+    c.epi.topk = topk_l;
+    c.epi.idx_offset = h->vocab_offset;
+    if (p.use_fp8[l]) {   // e4m3 operands; every tile keeps SPEC_MAX_TOPK candidates by approximate logit
+        c.A = ws + p.lay.state8;
+        c.B = h->head8[l];
+        c.epi.fp8 = 1;
+        c.epi.topk = SPEC_MAX_TOPK;
+        c.epi.row_scale = (const float *)(ws + p.lay.state8_scale);
+        c.epi.col_scale = h->head8_scale[l];
+    } else if (p.swapped[l]) {
+        c.A = w.head[l]; c.M = h->head_rows;
+        c.B = ws + p.lay.state[l]; c.N = p.N[l];
+        c.block_n = (p.N[l] + 15) / 16 * 16;
+        c.epi.mode = 3;
+    }
+    return c;
 }
 
 // State projection of level l as a tensor-core contraction: with few parent rows the weights take the
@@ -312,6 +367,7 @@ int spec_create(spec_handle_t *out, const spec_weights_t *w) {
     h->proj_block_n = 0;
     h->profile = 0;
     h->fp8_max_rows = 128;
+    h->swap_max_rows = 128;
     h->vp_rank = 0;
     h->vp_ranks = 1;
     h->vocab_offset = 0;
@@ -357,6 +413,10 @@ int spec_set_option(spec_handle_t h, int option, int value) {
         case SPEC_OPT_FP8_MAX_ROWS:
             if (value < 0 || value > (1 << 24)) return SPEC_ERR_INVALID_ARG;
             h->fp8_max_rows = value;
+            return SPEC_OK;
+        case SPEC_OPT_HEAD_SWAP_MAX_ROWS:
+            if (value < 0 || value > 128) return SPEC_ERR_INVALID_ARG;
+            h->swap_max_rows = value;
             return SPEC_OK;
         default:
             return SPEC_ERR_INVALID_ARG;
@@ -421,8 +481,13 @@ int spec_draft(spec_handle_t h, const void *ctx_state, const int32_t *last_tok, 
     const spec_weights_t &w = h->w;
     char *ws = (char *)workspace;
     int32_t *err = (int32_t *)(ws + p.lay.error_word);
-    rc = launch_draft_init(err, p.header_words, st);
-    if (rc != SPEC_OK) return rc;
+    // The header (error word, per-sequence counters) is cleared by the first kernel of the call: the level-0
+    // projection itself on the tensor-core path, a kernel of its own otherwise.
+    const bool clear_in_proj = h->gemm_impl == 0;
+    if (!clear_in_proj) {
+        rc = launch_draft_init(err, p.header_words, st);
+        if (rc != SPEC_OK) return rc;
+    }
 
     int nev = 0;
     h->prof_count = 0;
@@ -442,6 +507,7 @@ int spec_draft(spec_handle_t h, const void *ctx_state, const int32_t *last_tok, 
     const PruneArgs pa = make_prune_args(p, ws, topk);
     const bool fold_prune = !h->profile;
     bool proj_done = false;   // the projection of the level about to start ran with the previous head
+    bool mix_done = false;    // the states of the level about to start were written by the previous level's merge
     for (int l = 0; l < p.n; ++l) {
         const int rows = p.N[l];
         const int parent_rows = l == 0 ? B : p.N[l - 1];
@@ -453,7 +519,7 @@ int spec_draft(spec_handle_t h, const void *ctx_state, const int32_t *last_tok, 
         if (!proj_done) {
             if (h->gemm_impl == 0) {
                 const GemmCall c = proj_call(l);
-                rc = launch_gemm_tc_jobs(&c, 1, err, st);
+                rc = launch_gemm_tc_jobs(&c, 1, err, st, l == 0 ? err : nullptr, p.header_words);
             } else {
                 rc = run_gemm_store(h, parent_states, w.proj[l], parent_rows, w.d_inner, d_in_of(w, l),
                                     p.proj_block_n[l], P, err, st);
@@ -463,35 +529,25 @@ int spec_draft(spec_handle_t h, const void *ctx_state, const int32_t *last_tok, 
         SPEC_PROF_MARK();
         // gather + mix + LayerNorm + GELU -> bf16 state of every node of this level
         const bool fp8 = p.use_fp8[l];
-        MixArgs mx = make_mix_args(h, p, ws, last_tok, B, topk, l, err);
-        if (fp8) {   // the head of this level reads the states as e4m3
-            mx.S8_out = (uint8_t *)(ws + p.lay.state8);
-            mx.s8_scale = (float *)(ws + p.lay.state8_scale);
+        if (!mix_done) {
+            MixArgs mx = make_mix_args(h, p, ws, last_tok, B, topk, l, err);
+            if (fp8) {   // the head of this level reads the states as e4m3
+                mx.S8_out = (uint8_t *)(ws + p.lay.state8);
+                mx.s8_scale = (float *)(ws + p.lay.state8_scale);
+            }
+            rc = launch_mix_ln_gelu(mx, rows, st);
+            if (rc != SPEC_OK) return rc;
         }
-        rc = launch_mix_ln_gelu(mx, rows, st);
-        if (rc != SPEC_OK) return rc;
+        mix_done = false;
         SPEC_PROF_MARK();
         // vocabulary head with the fused per-tile top-k / log-sum-exp epilogue.  The next level's
         // projection needs nothing newer than this level's states either, so it rides in the same
         // launch: its weight tiles follow the head's through the same ring and one kernel boundary less
         // lies on the critical path (with per-kernel profiling it stays a launch of its own).
         proj_done = false;
-        if (h->gemm_impl == 0 && !h->profile && (l + 1 < p.n || fp8)) {
+        if (h->gemm_impl == 0 && !h->profile) {
             GemmCall c[2];
-            c[0].A = S; c[0].B = w.head[l]; c[0].M = rows; c[0].N = h->head_rows; c[0].Kd = w.d_inner;
-            c[0].block_n = p.lay.block_n[l];
-            c[0].epi = GemmEpilogue{};
-            c[0].epi.mode = 1;
-            c[0].epi.part_val = part_val; c[0].epi.part_idx = part_idx; c[0].epi.part_ms = part_ms;
-            c[0].epi.topk = topk[l];
-            if (fp8) {   // e4m3 operands; every tile keeps SPEC_MAX_TOPK candidates by approximate logit
-                c[0].A = ws + p.lay.state8;
-                c[0].B = h->head8[l];
-                c[0].epi.fp8 = 1;
-                c[0].epi.topk = SPEC_MAX_TOPK;
-                c[0].epi.row_scale = (const float *)(ws + p.lay.state8_scale);
-                c[0].epi.col_scale = h->head8_scale[l];
-            }
+            c[0] = make_head_call(h, p, ws, l, topk[l]);
             const bool pair = l + 1 < p.n;
             if (pair) c[1] = proj_call(l + 1);
             rc = launch_gemm_tc_jobs(c, pair ? 2 : 1, err, st);
@@ -525,7 +581,17 @@ int spec_draft(spec_handle_t h, const void *ctx_state, const int32_t *last_tok, 
             g.list_len = SPEC_MAX_TOPK;
             rc = launch_merge_rescore(g, w.head[l], S, rows, w.d_inner, w.V, st);
         } else {
-            rc = launch_merge_expand(g, rows, st);
+            rc = SPEC_ERR_SHAPE;
+            if (proj_done && topk[l] <= kFusedMixMaxChildren && !p.use_fp8[l + 1]) {
+                // the children's states in the same launch: their tokens are found here and their parent
+                // projection (this level's rows) ran with the head above.  Only for one or two children per
+                // row (the single-candidate chain above all): with more, a row's CTA would compute several
+                // states one after the other on one SM while a kernel of its own spreads them over the GPU
+                // (measured at the 13B shape: a draft 25 us slower with six and four children per CTA)
+                rc = launch_merge_mix(g, make_mix_args(h, p, ws, last_tok, B, topk, l + 1, err), rows, st);
+                mix_done = rc == SPEC_OK;
+            }
+            if (rc == SPEC_ERR_SHAPE) rc = launch_merge_expand(g, rows, st);
         }
         if (rc != SPEC_OK) return rc;
         SPEC_PROF_MARK();
@@ -578,15 +644,12 @@ int spec_draft_vp_local(spec_handle_t h, int level, const void *ctx_state, const
     if (!workspace || ((uintptr_t)workspace % kWsAlign) != 0 || workspace_bytes < p.lay.total_bytes)
         return SPEC_ERR_WORKSPACE;
     cudaStream_t st = (cudaStream_t)cuda_stream;
-    const spec_weights_t &w = h->w;
     char *ws = (char *)workspace;
     int32_t *err = (int32_t *)(ws + p.lay.error_word);
     const int l = level, rows = p.N[l];
     if (l == 0) {   // the first step of a draft clears the header and projects the context states
-        rc = launch_draft_init(err, p.header_words, st);
-        if (rc != SPEC_OK) return rc;
         const GemmCall c = make_proj_call(h, p, ws, ctx_state, B, 0);
-        rc = launch_gemm_tc_jobs(&c, 1, err, st);
+        rc = launch_gemm_tc_jobs(&c, 1, err, st, err, p.header_words);
         if (rc != SPEC_OK) return rc;
     }
     const MixArgs mx = make_mix_args(h, p, ws, last_tok, B, topk, l, err);
@@ -595,15 +658,7 @@ int spec_draft_vp_local(spec_handle_t h, int level, const void *ctx_state, const
     // this rank's vocabulary rows only; token ids leave the epilogue already offset.  The next level's
     // projection (replicated on every rank) rides in the same launch as in spec_draft.
     GemmCall c[2];
-    c[0] = GemmCall{};
-    c[0].A = ws + p.lay.state[l]; c[0].B = w.head[l]; c[0].M = rows; c[0].N = h->head_rows; c[0].Kd = w.d_inner;
-    c[0].block_n = p.lay.block_n[l];
-    c[0].epi.mode = 1;
-    c[0].epi.part_val = (float *)(ws + p.lay.part_val);
-    c[0].epi.part_idx = (int32_t *)(ws + p.lay.part_idx);
-    c[0].epi.part_ms = (float *)(ws + p.lay.part_ms);
-    c[0].epi.topk = topk[l];
-    c[0].epi.idx_offset = h->vocab_offset;
+    c[0] = make_head_call(h, p, ws, l, topk[l]);
     const bool pair = l + 1 < p.n;
     if (pair) c[1] = make_proj_call(h, p, ws, ctx_state, B, l + 1);
     rc = launch_gemm_tc_jobs(c, pair ? 2 : 1, err, st);
@@ -701,8 +756,7 @@ int spec_poll_error(void *workspace, void *cuda_stream) {
 
 size_t spec_head_workspace_bytes(spec_handle_t h, int rows, int topk) {
     if (!h || rows <= 0 || topk < 1 || topk > SPEC_MAX_TOPK || h->vp_ranks > 1) return 0;
-    const int bn = head_block_n_for(h, rows);
-    const size_t units = (size_t)rows * ((h->w.V + bn - 1) / bn);
+    const size_t units = (size_t)rows * head_parts_for(h, rows, head_swapped_for(h, rows), nullptr);
     size_t off = kWsAlign;
     off = align_up(off + sizeof(float) * units * SPEC_MAX_TOPK, kWsAlign);
     off = align_up(off + sizeof(int32_t) * units * SPEC_MAX_TOPK, kWsAlign);
@@ -730,8 +784,8 @@ static int head_topk_impl(spec_handle_t h, int level, const void *states, int ro
     const size_t need = spec_head_workspace_bytes(h, rows, topk);
     if (!workspace || ((uintptr_t)workspace % kWsAlign) != 0 || workspace_bytes < need) return SPEC_ERR_WORKSPACE;
     cudaStream_t st = (cudaStream_t)cuda_stream;
-    const int bn = head_block_n_for(h, rows);
-    const int n_tiles = (h->w.V + bn - 1) / bn;
+    int bn = 0;
+    const int n_tiles = head_parts_for(h, rows, head_swapped_for(h, rows), &bn);
     const size_t units = (size_t)rows * n_tiles;
     char *ws = (char *)workspace;
     int32_t *err = (int32_t *)ws;

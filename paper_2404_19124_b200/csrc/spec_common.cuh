@@ -93,7 +93,10 @@ int launch_verify_early(const int32_t *cand_tok, const void *base_logits, int dt
 // C[M, N] = A[M, Kd] * B[N, Kd]^T, A and B bf16 row-major (K-major), fp32 accumulation in TMEM.
 struct GemmEpilogue {
     int mode;          // 0: store fp32 C; 1: per-row partial top-k + (max, sum-exp) per tile;
-                       // 2: split-K partials stored transposed, out[split][n][m]
+                       // 2: split-K partials stored transposed, out[split][n][m];
+                       // 3: vocabulary head with the operands swapped (A = head weights [V, Kd], B = states
+                       //    [nodes <= 128, Kd]): per node and (CTA, segment) one partial top-k list and
+                       //    (max, sum-exp) in the mode-1 arrays, n_parts lists per node
     float *out;        // mode 0: [M, N] row-major; mode 2: [splits][N][ldc]
     int ldc;           // mode 0 / 2: leading dimension of out
     int splits;        // mode 2: number of K ranges, each handled by its own tile
@@ -105,8 +108,13 @@ struct GemmEpilogue {
     int fp8;           // operands are e4m3 bytes instead of bf16; mode 1 then multiplies every accumulator by
                        // row_scale[m] * col_scale[n] before the selection
     const float *row_scale, *col_scale;
-    int idx_offset;    // mode 1: added to every column index written to part_idx (first vocabulary row of a shard)
+    int idx_offset;    // mode 1 / 3: added to every token id written to part_idx (first vocabulary row of a shard)
+    int segs;          // mode 3: threads that share one node's column (swapped_head_segs)
+    int n_parts;       // mode 3: partial lists per node = CTAs the tiles are dealt to * segs (swapped_head_parts)
 };
+// Mode 3 bookkeeping, the same on the host (workspace sizing, merge) and in the launch.
+int swapped_head_segs(int nodes);
+int swapped_head_parts(int nodes, int vocab_rows);
 int choose_block_n(int M, int N, int num_sm, bool tensor_bound_pref);
 int launch_gemm_tc(const void *A, const void *B, int M, int N, int Kd, int block_n, const GemmEpilogue &epi,
                    int32_t *err, cudaStream_t st);
@@ -116,7 +124,10 @@ struct GemmCall {
     int M, N, Kd, block_n;
     GemmEpilogue epi;
 };
-int launch_gemm_tc_jobs(const GemmCall *calls, int n_calls, int32_t *err, cudaStream_t st);
+// `clear` / `clear_words`: int32 words that CTA 0 zeroes once the preceding grid has completed (the first
+// kernel of a draft clears the workspace header this way); null: nothing.
+int launch_gemm_tc_jobs(const GemmCall *calls, int n_calls, int32_t *err, cudaStream_t st, int32_t *clear = nullptr,
+                        int clear_words = 0);
 
 // ---- debug CUDA-core GEMM (gemm_simt.cu) ------------------------------------------------
 int launch_gemm_simt(const void *A, const void *B, int M, int N, int Kd, float *C, int ldc, cudaStream_t st);
@@ -176,6 +187,8 @@ int launch_merge_rescore(const MergeArgs &g, const void *W, const void *S, int r
 int launch_draft_init(int32_t *hdr, int words, cudaStream_t st);
 int launch_mix_ln_gelu(const MixArgs &m, int rows, cudaStream_t st);
 int launch_merge_expand(const MergeArgs &g, int rows, cudaStream_t st);
+// merge of one level + mix of the next in one kernel; SPEC_ERR_SHAPE: shape not covered, launch them separately
+int launch_merge_mix(const MergeArgs &g, const MixArgs &m, int rows, cudaStream_t st);
 // Cross-shard merge of a vocabulary-parallel head.  Slot g (g < n_ranks, `slot_bytes` apart, starting at
 // `slots`) holds rank g's raw lists: fp32 values [rows, topk], int32 token ids [rows, topk], fp32 lse [rows].
 // Children of every row: the topk best of the n_ranks*topk entries (value desc, token id asc) with

@@ -9,6 +9,12 @@
 //               commits to the slot's "empty" barrier and, per tile, to "accumulator full"
 //   warps 2-5   epilogue: tcgen05.ld of 32 columns at a time, one thread per accumulator row
 // Two accumulator slots in TMEM let the epilogue of tile i overlap the MMAs of tile i + 1.
+// Epilogue modes: 0 plain fp32 store; 1 per-row partial top-k + (max, sum-exp) with one thread per accumulator
+// row; 2 split-K partials stored transposed (operands swapped: weights on the 128-row side); 3 the vocabulary
+// head with the operands swapped (levels of at most 128 nodes: the MMA work then follows the number of nodes
+// instead of being padded to 128 rows): the accumulator tile [128 vocabulary rows x nodes] is transposed
+// through shared memory and every node's column is scanned by its own threads, which keep one running
+// top-k list and (max, sum-exp) pair for all tiles of the CTA.
 // A "job" is one contraction; its tiles (m fastest, then n, then the K split) are dealt round-robin to
 // the CTAs of the grid, and each role walks the jobs it is given in the same order, carrying its ring
 // position from one job to the next.  Every wait is bounded: when one runs out the CTA records
@@ -32,6 +38,9 @@ constexpr int kABytes = kBlockM * kSlabBytes;
 constexpr int kSmemLimit = 222 * 1024; // leaves room on the SM for the small kernels that overlap with a GEMM
 constexpr uint32_t kSpinFast = 1u << 14;
 constexpr uint32_t kSpinMax = 1u << 24;
+constexpr int kTPitch = kBlockM + 4;   // floats between the columns of the transposed tile (mode 3): rows of four
+                                       // floats stay 16-byte aligned and eight neighbouring columns hit 32 banks
+constexpr int kSwapMaxSegs = 8;        // most threads that share one node's column in the mode-3 scan
 
 struct __align__(8) Barriers {
     uint64_t full[kMaxStages];
@@ -40,6 +49,7 @@ struct __align__(8) Barriers {
     uint64_t acc_empty[2];
     uint32_t tmem_base;
     volatile int abort_flag;
+    volatile int epi_ok;        // mode 3: the epilogue leader's verdict on its wait, read by the other epilogue warps
 };
 
 // One contraction as the kernels see it.
@@ -49,7 +59,11 @@ struct GemmJob {
     int splits, kb_per_split;   // split-K: tile = (m_tile, n_tile, split), split slowest
     int fp8;                    // 0: bf16 operands (kind::f16); 1: e4m3 operands (kind::f8f6f4); fp32 accumulation either way
     int w_is_a;                 // 1: A holds the weights (no kernel writes them), B the states; 0: the reverse
-    int first_cta;              // CTA that takes tile 0; tile t goes to CTA (first_cta + t) mod grid
+    int first_cta;              // CTA that takes tile 0; tile t goes to CTA (first_cta + t mod deal_ctas) mod grid
+    int deal_ctas;              // CTAs the tiles are dealt to, consecutive from first_cta (0: the whole grid)
+    int rows_per_cta;           // mode 3: A rows (vocabulary rows) of every CTA of the deal, a multiple of 8: CTA c
+                                // of the deal takes rows [c * rows_per_cta, (c + 1) * rows_per_cta) as 128-row tiles
+                                // plus one shorter tile, so that every CTA streams the same number of bytes
     GemmEpilogue epi;
 };
 
@@ -61,6 +75,7 @@ struct Pipe {
     int stages;
     uint32_t slot_bytes;
     int acc_stride;        // TMEM columns between the two accumulator slots
+    float *tbuf;           // mode 3: transposed accumulator tile, [nodes][kTPitch] floats (null when not used)
     int32_t *err;
 };
 
@@ -160,6 +175,20 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32]) {
     for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
 }
 
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, float (&v)[16]) {
+    uint32_t r[16];
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+        : "r"(taddr)
+        : "memory");
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+    for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
+}
+
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 
@@ -173,10 +202,11 @@ __device__ __forceinline__ float ex2_approx(float x) {
 // Called by all threads.  Initialises the barriers, allocates `tmem_cols` TMEM columns (a power of two,
 // at least 32) and returns the pipe description.
 __device__ __forceinline__ Pipe pipe_setup(uint8_t *smem_raw, int stages, uint32_t slot_bytes, int tmem_cols,
-                                           int acc_stride, int32_t *err) {
+                                           int acc_stride, uint32_t tbuf_bytes, int32_t *err) {
     Pipe pp;
     pp.tiles = (uint8_t *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);   // swizzled tiles: 1024-byte aligned
-    pp.bars = (Barriers *)(pp.tiles + (size_t)stages * slot_bytes);
+    pp.tbuf = tbuf_bytes ? (float *)(pp.tiles + (size_t)stages * slot_bytes) : nullptr;
+    pp.bars = (Barriers *)(pp.tiles + (size_t)stages * slot_bytes + tbuf_bytes);
     pp.stages = stages;
     pp.slot_bytes = slot_bytes;
     pp.acc_stride = acc_stride;
@@ -192,6 +222,7 @@ __device__ __forceinline__ Pipe pipe_setup(uint8_t *smem_raw, int stages, uint32
             mbar_init(&pp.bars->acc_empty[a], 4);   // one arrival per epilogue warp
         }
         pp.bars->abort_flag = 0;
+        pp.bars->epi_ok = 1;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
@@ -224,8 +255,60 @@ __device__ __forceinline__ void pipe_teardown(const Pipe &pp, int tmem_cols) {
 __device__ __forceinline__ int slab_elems(const GemmJob &j) { return j.fp8 ? kSlabBytes : kSlabBytes / 2; }
 __device__ __forceinline__ int num_k_blocks(const GemmJob &j) { return (j.Kd + slab_elems(j) - 1) / slab_elems(j); }
 
-__device__ __forceinline__ int first_tile_of(const GemmJob &j) {
+// The tiles of job j that this CTA takes, as a walk  t = first, first + step, ... < end.
+// Modes 0-2: tile index = (split, n_tile, m_tile) with m fastest, dealt round-robin over the CTAs of the deal.
+// Mode 3: the CTA's own run of A rows cut into 128-row tiles; t counts them from 0.
+struct TileWalk { int first, end, step, rel; };
+struct TilePos {
+    int a_row, b_row;    // first row of the A box and of the B box
+    int kb0, kb1;        // K blocks [kb0, kb1)
+    int a_rows;          // rows of the A box (mode 3: the last tile of a CTA may be shorter)
+    int split, m_tile, n_tile;
+};
+
+__device__ __forceinline__ int cta_rel(const GemmJob &j) {
     return (int)((blockIdx.x + gridDim.x - (unsigned)j.first_cta % gridDim.x) % gridDim.x);
+}
+
+__device__ __forceinline__ TileWalk walk_of(const GemmJob &j) {
+    TileWalk w;
+    w.rel = cta_rel(j);
+    if (j.epi.mode == 3) {
+        int rows = 0;
+        if (w.rel < j.deal_ctas) rows = min(j.M - w.rel * j.rows_per_cta, j.rows_per_cta);
+        w.first = 0;
+        w.end = rows > 0 ? (rows + kBlockM - 1) / kBlockM : 0;
+        w.step = 1;
+    } else {
+        w.step = j.deal_ctas > 0 ? j.deal_ctas : (int)gridDim.x;
+        w.end = j.m_tiles * j.n_tiles * j.splits;
+        w.first = w.rel < w.step ? w.rel : w.end;
+    }
+    return w;
+}
+
+__device__ __forceinline__ TilePos pos_of(const GemmJob &j, const TileWalk &w, int t) {
+    TilePos q;
+    const int num_kb = (j.Kd + (j.fp8 ? kSlabBytes : kSlabBytes / 2) - 1) / (j.fp8 ? kSlabBytes : kSlabBytes / 2);
+    if (j.epi.mode == 3) {
+        q.a_row = w.rel * j.rows_per_cta + t * kBlockM;
+        q.b_row = 0;
+        q.kb0 = 0; q.kb1 = num_kb;
+        q.a_rows = (t + 1) * kBlockM <= j.rows_per_cta ? kBlockM : j.rows_per_cta - t * kBlockM;
+        q.split = 0; q.m_tile = t; q.n_tile = 0;
+    } else {
+        const int mn_tiles = j.m_tiles * j.n_tiles;
+        q.split = t / mn_tiles;
+        const int mn = t - q.split * mn_tiles;
+        q.m_tile = mn % j.m_tiles;
+        q.n_tile = mn / j.m_tiles;
+        q.a_row = q.m_tile * kBlockM;
+        q.b_row = q.n_tile * j.block_n;
+        q.kb0 = q.split * j.kb_per_split;
+        q.kb1 = min(num_kb, q.kb0 + j.kb_per_split);
+        q.a_rows = kBlockM;
+    }
+    return q;
 }
 
 __device__ __forceinline__ void advance(const Pipe &pp, RingPos &rp) {
@@ -240,37 +323,36 @@ __device__ __forceinline__ void advance(const Pipe &pp, RingPos &rp) {
 // loads nor waits.  `issued` counts slots filled since the kernel started (for the abort path).
 template <typename DepWait>
 __device__ __forceinline__ bool produce_job(const Pipe &pp, const GemmJob &j, const CUtensorMap *tmap_a,
-                                            const CUtensorMap *tmap_b, RingPos &rp, int &issued, DepWait dep_wait) {
-    const int num_kb = num_k_blocks(j), ke = slab_elems(j);
-    const int mn_tiles = j.m_tiles * j.n_tiles;
-    const int num_tiles = mn_tiles * j.splits;
-    const uint32_t tx = (uint32_t)kABytes + (uint32_t)j.block_n * kSlabBytes;
-    const int first = first_tile_of(j);
-    if (first >= num_tiles) return true;
+                                            const CUtensorMap *tmap_a_short, const CUtensorMap *tmap_b, RingPos &rp,
+                                            int &issued, DepWait dep_wait) {
+    const int ke = slab_elems(j);
+    const uint32_t b_bytes = (uint32_t)j.block_n * kSlabBytes;
+    const TileWalk w = walk_of(j);
+    if (w.first >= w.end) return true;
     Barriers *bars = pp.bars;
     int n_pre = 0;
     {
-        const int split = first / mn_tiles, mn = first - split * mn_tiles;
-        const int m_tile = mn % j.m_tiles, n_tile = mn / j.m_tiles;
-        const int kb0 = split * j.kb_per_split, kb1 = min(num_kb, kb0 + j.kb_per_split);
-        n_pre = min(pp.stages, kb1 - kb0);
+        const TilePos t0 = pos_of(j, w, w.first);
+        const CUtensorMap *ma = t0.a_rows == kBlockM ? tmap_a : tmap_a_short;
+        const uint32_t tx = (uint32_t)t0.a_rows * kSlabBytes + b_bytes;
+        n_pre = min(pp.stages, t0.kb1 - t0.kb0);
         RingPos q = rp;
         for (int i = 0; i < n_pre; ++i) {
             if (!mbar_wait(&bars->empty[q.stage], q.phase ^ 1u, bars, pp.err)) return false;
             uint8_t *sa = pp.tiles + (size_t)q.stage * pp.slot_bytes;
             mbar_arrive_expect_tx(&bars->full[q.stage], tx);
-            if (j.w_is_a) tma_load_2d(sa, tmap_a, (kb0 + i) * ke, m_tile * kBlockM, &bars->full[q.stage]);
-            else tma_load_2d(sa + kABytes, tmap_b, (kb0 + i) * ke, n_tile * j.block_n, &bars->full[q.stage]);
+            if (j.w_is_a) tma_load_2d(sa, ma, (t0.kb0 + i) * ke, t0.a_row, &bars->full[q.stage]);
+            else tma_load_2d(sa + kABytes, tmap_b, (t0.kb0 + i) * ke, t0.b_row, &bars->full[q.stage]);
             advance(pp, q);
         }
     }
     if (!dep_wait()) return false;
     int done = 0;   // k blocks of this job handled so far
-    for (int tile = first; tile < num_tiles; tile += gridDim.x) {
-        const int split = tile / mn_tiles, mn = tile - split * mn_tiles;
-        const int m_tile = mn % j.m_tiles, n_tile = mn / j.m_tiles;
-        const int kb0 = split * j.kb_per_split, kb1 = min(num_kb, kb0 + j.kb_per_split);
-        for (int kb = kb0; kb < kb1; ++kb) {
+    for (int tile = w.first; tile < w.end; tile += w.step) {
+        const TilePos t = pos_of(j, w, tile);
+        const CUtensorMap *ma = t.a_rows == kBlockM ? tmap_a : tmap_a_short;
+        const uint32_t tx = (uint32_t)t.a_rows * kSlabBytes + b_bytes;
+        for (int kb = t.kb0; kb < t.kb1; ++kb) {
             uint8_t *sa = pp.tiles + (size_t)rp.stage * pp.slot_bytes;
             uint8_t *sb = sa + kABytes;
             const bool prefetched = done < n_pre;   // the weights of this slot are already on their way
@@ -278,8 +360,8 @@ __device__ __forceinline__ bool produce_job(const Pipe &pp, const GemmJob &j, co
                 if (!mbar_wait(&bars->empty[rp.stage], rp.phase ^ 1u, bars, pp.err)) return false;
                 mbar_arrive_expect_tx(&bars->full[rp.stage], tx);
             }
-            if (!prefetched || !j.w_is_a) tma_load_2d(sa, tmap_a, kb * ke, m_tile * kBlockM, &bars->full[rp.stage]);
-            if (!prefetched || j.w_is_a) tma_load_2d(sb, tmap_b, kb * ke, n_tile * j.block_n, &bars->full[rp.stage]);
+            if (!prefetched || !j.w_is_a) tma_load_2d(sa, ma, kb * ke, t.a_row, &bars->full[rp.stage]);
+            if (!prefetched || j.w_is_a) tma_load_2d(sb, tmap_b, kb * ke, t.b_row, &bars->full[rp.stage]);
             ++done;
             ++issued;
             advance(pp, rp);
@@ -342,21 +424,19 @@ __device__ __forceinline__ void umma_k_block(uint32_t tmem_d, uint32_t lo_a, uin
 template <bool kFp8>
 __device__ __forceinline__ bool mma_job_kind(const Pipe &pp, const GemmJob &j, RingPos &rp, AccPos &ap) {
     static_assert(kSlabBytes / kUmmaBytes == 4, "umma_k_block issues four MMAs");
-    const int num_kb = num_k_blocks(j);
-    const int mn_tiles = j.m_tiles * j.n_tiles;
-    const int num_tiles = mn_tiles * j.splits;
     const uint32_t idesc = make_instr_desc(kBlockM, j.block_n, kFp8);
     const uint32_t desc_hi = (uint32_t)(make_smem_desc(0) >> 32);
     const uint32_t lo_base = (smem_u32(pp.tiles) & 0x3ffffu) >> 4, lo_slot = pp.slot_bytes >> 4;
     Barriers *bars = pp.bars;
-    for (int tile = first_tile_of(j); tile < num_tiles; tile += gridDim.x) {
+    const TileWalk w = walk_of(j);
+    for (int tile = w.first; tile < w.end; tile += w.step) {
         if (!mbar_wait(&bars->acc_empty[ap.acc], ap.phase ^ 1u, bars, pp.err)) return false;
         tc_fence_after();
         const uint32_t tmem_d = pp.tmem_base + (uint32_t)(ap.acc * pp.acc_stride);
-        const int split = tile / mn_tiles;
-        const int kb0 = split * j.kb_per_split, kb1 = min(num_kb, kb0 + j.kb_per_split);
+        const TilePos t = pos_of(j, w, tile);
         uint32_t acc = 0u;
-        for (int kb = kb0; kb < kb1; ++kb) {
+        // (a short A box leaves the rest of the 128 rows as they were: those accumulator lanes are never read)
+        for (int kb = t.kb0; kb < t.kb1; ++kb) {
             if (!mbar_wait(&bars->full[rp.stage], rp.phase, bars, pp.err)) return false;
             tc_fence_after();
             const uint32_t lo_a = lo_base + (uint32_t)rp.stage * lo_slot;
@@ -506,17 +586,237 @@ __device__ __forceinline__ void epilogue_topk(const GemmJob &p, uint32_t taddr, 
     }
 }
 
+// ---- epilogue, mode 3 (operands swapped: TMEM lanes are vocabulary rows, columns are nodes) ----------
+// What one scan thread carries from tile to tile: the running (max, sum-exp) of its share of a node's
+// logits and the best SPEC_MAX_TOPK of them, best first by (value desc, token id asc).
+struct SwapRun {
+    float m, s;
+    float tv[SPEC_MAX_TOPK];
+    int ti[SPEC_MAX_TOPK];
+};
+
+__device__ __forceinline__ bool cand_better(float v, int i, float w, int j) { return v > w || (v == w && i < j); }
+
+// Branch-free insertion into the sorted list: slot j takes its left neighbour when the newcomer beats that
+// neighbour, the newcomer when it beats only slot j, and keeps its entry otherwise.
+__device__ __forceinline__ void list_insert(SwapRun &r, float x, int id) {
+    bool beats[SPEC_MAX_TOPK];
+#pragma unroll
+    for (int j = 0; j < SPEC_MAX_TOPK; ++j) beats[j] = cand_better(x, id, r.tv[j], r.ti[j]);
+#pragma unroll
+    for (int j = SPEC_MAX_TOPK - 1; j > 0; --j) {
+        r.tv[j] = beats[j - 1] ? r.tv[j - 1] : (beats[j] ? x : r.tv[j]);
+        r.ti[j] = beats[j - 1] ? r.ti[j - 1] : (beats[j] ? id : r.ti[j]);
+    }
+    r.tv[0] = beats[0] ? x : r.tv[0];
+    r.ti[0] = beats[0] ? id : r.ti[0];
+}
+
+__device__ __forceinline__ void epi_bar_sync() { asm volatile("bar.sync 1, %0;" ::"n"(kEpilogueThreads) : "memory"); }
+
+// One thread scans `len` (a multiple of 16) consecutive logits of one node in the transposed tile: `col`
+// points at the first, `valid` of them are real vocabulary rows (the rest hold -inf), `idx0` is the token id
+// of the first.  Pass 1: online (max, sum-exp) and the kCap largest values (min/max network).  Pass 2: the
+// entries that reach the topk-th largest value, ties in ascending token order, exactly topk of them, are
+// inserted into the running list.
+template <int kCap>
+__device__ __forceinline__ void swap_scan_tile(const float *col, int len, int valid, int idx0, int topk, SwapRun &r) {
+    constexpr float kLog2e = 1.4426950408889634f;
+    float best[kCap];
+#pragma unroll
+    for (int j = 0; j < kCap; ++j) best[j] = -INFINITY;
+    for (int c = 0; c < len; c += 16) {
+        float v[16];
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            const float4 f = *(const float4 *)(col + c + 4 * q);
+            v[4 * q] = f.x; v[4 * q + 1] = f.y; v[4 * q + 2] = f.z; v[4 * q + 3] = f.w;
+        }
+        float cm0 = fmaxf(v[0], v[1]), cm1 = fmaxf(v[2], v[3]);
+#pragma unroll
+        for (int i = 4; i < 16; i += 2) {
+            cm0 = fmaxf(cm0, v[i]);
+            cm1 = fmaxf(cm1, v[i + 1]);
+        }
+        const float cm = fmaxf(cm0, cm1);
+        if (cm > r.m) {
+            r.s *= ex2_approx((r.m - cm) * kLog2e);
+            r.m = cm;
+        }
+        const float ms = r.m * kLog2e;
+        float s0 = 0.0f, s1 = 0.0f, s2 = 0.0f, s3 = 0.0f;
+#pragma unroll
+        for (int i = 0; i < 16; i += 4) {
+            s0 += ex2_approx(fmaf(v[i], kLog2e, -ms));
+            s1 += ex2_approx(fmaf(v[i + 1], kLog2e, -ms));
+            s2 += ex2_approx(fmaf(v[i + 2], kLog2e, -ms));
+            s3 += ex2_approx(fmaf(v[i + 3], kLog2e, -ms));
+        }
+        if (r.m > -INFINITY) r.s += (s0 + s1) + (s2 + s3);
+#pragma unroll
+        for (int i = 0; i < 16; ++i) {
+            const float x = v[i];
+#pragma unroll
+            for (int j = kCap - 1; j > 0; --j) best[j] = fmaxf(best[j], fminf(best[j - 1], x));
+            best[0] = fmaxf(best[0], x);
+        }
+    }
+    float thr = best[0];
+#pragma unroll
+    for (int j = 1; j < kCap; ++j)
+        if (j < topk) thr = best[j];
+    int above = 0;
+#pragma unroll
+    for (int j = 0; j < kCap; ++j)
+        if (j < topk && best[j] > thr) ++above;
+    int eq_left = topk - above;
+    for (int c = 0; c < len; c += 16) {
+        uint32_t mask = 0;
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            const float4 f = *(const float4 *)(col + c + 4 * q);
+            mask |= (f.x >= thr ? 1u : 0u) << (4 * q);
+            mask |= (f.y >= thr ? 1u : 0u) << (4 * q + 1);
+            mask |= (f.z >= thr ? 1u : 0u) << (4 * q + 2);
+            mask |= (f.w >= thr ? 1u : 0u) << (4 * q + 3);
+        }
+        const int left = valid - c;
+        if (left < 16) mask &= left > 0 ? ((1u << left) - 1u) : 0u;
+        while (mask) {   // ascending token ids; a handful of iterations per tile
+            const int bpos = __ffs(mask) - 1;
+            mask &= mask - 1;
+            const float x = col[c + bpos];
+            const bool gt = x > thr;
+            if (gt || eq_left > 0) {
+                if (!gt) --eq_left;
+                list_insert(r, x, idx0 + c + bpos);
+            }
+        }
+    }
+}
+
+// The better eight of two lists that are both sorted best first: "the better of a[i] and b[7 - i]" keeps the
+// best eight as a bitonic sequence, which three compare-exchange stages sort.
+__device__ __forceinline__ void merge_sorted8(SwapRun &r, const float (&ov)[SPEC_MAX_TOPK], const int (&oi)[SPEC_MAX_TOPK]) {
+    constexpr int kT = SPEC_MAX_TOPK;
+    static_assert(kT == 8, "three stages sort eight entries");
+#pragma unroll
+    for (int j = 0; j < kT; ++j) {
+        if (cand_better(ov[kT - 1 - j], oi[kT - 1 - j], r.tv[j], r.ti[j])) {
+            r.tv[j] = ov[kT - 1 - j];
+            r.ti[j] = oi[kT - 1 - j];
+        }
+    }
+#pragma unroll
+    for (int stride = kT / 2; stride > 0; stride >>= 1) {
+#pragma unroll
+        for (int j = 0; j < kT; ++j) {
+            if ((j & stride) == 0 && cand_better(r.tv[j + stride], r.ti[j + stride], r.tv[j], r.ti[j])) {
+                const float fv = r.tv[j]; r.tv[j] = r.tv[j + stride]; r.tv[j + stride] = fv;
+                const int fi = r.ti[j]; r.ti[j] = r.ti[j + stride]; r.ti[j + stride] = fi;
+            }
+        }
+    }
+}
+
+// Epilogue warps of a mode-3 job.  Per tile: the leader waits for the accumulator and tells the others
+// (so that all 128 threads take the same path into the barriers below, also when the wait gives up); every
+// thread copies its vocabulary row of the accumulator into the transposed tile in shared memory; after a
+// barrier the accumulator slot is released and the scan threads (P per node, each 128 / P rows of the tile)
+// fold their segment into their running list.  The barrier at the top of the next tile keeps the transposed
+// tile intact until every scan of this one is done.  After the last tile the P threads of a node (neighbouring
+// lanes) combine their lists and (max, sum-exp) pairs with shuffles and the first of them writes the node's
+// partial slot of this CTA.
+__device__ __forceinline__ bool epilogue_job_swapped(const Pipe &pp, const GemmJob &j, AccPos &ap) {
+    constexpr float kLog2e = 1.4426950408889634f;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int quarter = warp & 3;                    // TMEM lane quarter this warp may read
+    const int vrow = quarter * 32 + lane;            // vocabulary row of the tile held by this thread's TMEM lane
+    const int u = (int)threadIdx.x - (kThreads - kEpilogueThreads);
+    const int nodes = j.N, P = j.epi.segs, len = kBlockM / P;
+    const int node = u / P, seg = u - node * P;
+    const bool scans = node < nodes;
+    const int topk = j.epi.topk;
+    Barriers *bars = pp.bars;
+    SwapRun run;
+    run.m = -INFINITY;
+    run.s = 0.0f;
+#pragma unroll
+    for (int q = 0; q < SPEC_MAX_TOPK; ++q) {
+        run.tv[q] = -INFINITY;
+        run.ti[q] = 0x7fffffff;
+    }
+    const TileWalk w = walk_of(j);
+    const int row_end = min(j.M, (w.rel + 1) * j.rows_per_cta);   // the next CTA's rows start here
+    for (int tile = w.first; tile < w.end; tile += w.step) {
+        if (u == 0) bars->epi_ok = mbar_wait(&bars->acc_full[ap.acc], ap.phase, bars, pp.err) ? 1 : 0;
+        epi_bar_sync();
+        if (!bars->epi_ok) return false;
+        tc_fence_after();
+        const uint32_t taddr = pp.tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(ap.acc * pp.acc_stride);
+        const int row0 = w.rel * j.rows_per_cta + tile * kBlockM;   // vocabulary row of TMEM lane 0
+        const bool v_ok = row0 + vrow < row_end;
+        for (int c = 0; c < nodes; c += 16) {
+            float v[16];
+            tmem_ld16(taddr + c, v);
+#pragma unroll
+            for (int i = 0; i < 16; ++i)
+                if (c + i < nodes) pp.tbuf[(c + i) * kTPitch + vrow] = v_ok ? v[i] : -INFINITY;
+        }
+        tc_fence_before();
+        epi_bar_sync();
+        if (lane == 0) mbar_arrive(&bars->acc_empty[ap.acc]);
+        if (++ap.acc == 2) { ap.acc = 0; ap.phase ^= 1u; }
+        if (scans) {
+            const int seg_row = row0 + seg * len;            // first vocabulary row of this thread's segment
+            int valid = row_end - seg_row;
+            valid = valid < 0 ? 0 : (valid > len ? len : valid);
+            const float *col = pp.tbuf + node * kTPitch + seg * len;
+            if (topk <= 4) swap_scan_tile<4>(col, len, valid, seg_row + j.epi.idx_offset, topk, run);
+            else swap_scan_tile<SPEC_MAX_TOPK>(col, len, valid, seg_row + j.epi.idx_offset, topk, run);
+        }
+    }
+    if (w.first >= w.end) return true;
+    // the P neighbouring lanes of a node fold their results (every lane of the warp takes part in the shuffles)
+    for (int off = 1; off < P; off <<= 1) {
+        float ov[SPEC_MAX_TOPK];
+        int oi[SPEC_MAX_TOPK];
+#pragma unroll
+        for (int q = 0; q < SPEC_MAX_TOPK; ++q) {
+            ov[q] = __shfl_xor_sync(0xffffffffu, run.tv[q], off);
+            oi[q] = __shfl_xor_sync(0xffffffffu, run.ti[q], off);
+        }
+        const float om = __shfl_xor_sync(0xffffffffu, run.m, off), os = __shfl_xor_sync(0xffffffffu, run.s, off);
+        merge_sorted8(run, ov, oi);
+        const float nm = fmaxf(run.m, om);
+        if (nm > -INFINITY)
+            run.s = run.s * ex2_approx((run.m - nm) * kLog2e) + os * ex2_approx((om - nm) * kLog2e);
+        run.m = nm;
+    }
+    if (scans && seg == 0) {
+        const size_t slot = (size_t)node * j.epi.n_parts + (size_t)w.rel;
+        float4 *pv = (float4 *)(j.epi.part_val + slot * SPEC_MAX_TOPK);
+        int4 *pi = (int4 *)(j.epi.part_idx + slot * SPEC_MAX_TOPK);
+        pv[0] = make_float4(run.tv[0], run.tv[1], run.tv[2], run.tv[3]);
+        pv[1] = make_float4(run.tv[4], run.tv[5], run.tv[6], run.tv[7]);
+        pi[0] = make_int4(run.ti[0], run.ti[1], run.ti[2], run.ti[3]);
+        pi[1] = make_int4(run.ti[4], run.ti[5], run.ti[6], run.ti[7]);
+        *(float2 *)(j.epi.part_ms + 2 * slot) = make_float2(run.m, run.s);
+    }
+    return true;
+}
+
 // ---- epilogue warps (warps 2-5, all lanes) ----------------------------------------------------------
 __device__ __forceinline__ bool epilogue_job(const Pipe &pp, const GemmJob &j, AccPos &ap) {
+    if (j.epi.mode == 3) return epilogue_job_swapped(pp, j, ap);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int quarter = warp & 3;               // TMEM lane quarter this warp may read
     const int row_in_tile = quarter * 32 + lane;
-    const int mn_tiles = j.m_tiles * j.n_tiles;
-    const int num_tiles = mn_tiles * j.splits;
     Barriers *bars = pp.bars;
-    for (int tile = first_tile_of(j); tile < num_tiles; tile += gridDim.x) {
-        const int split = tile / mn_tiles, mn = tile - split * mn_tiles;
-        const int m_tile = mn % j.m_tiles, n_tile = mn / j.m_tiles;
+    const TileWalk w = walk_of(j);
+    for (int tile = w.first; tile < w.end; tile += w.step) {
+        const TilePos t = pos_of(j, w, tile);
+        const int split = t.split, m_tile = t.m_tile, n_tile = t.n_tile;
         if (!mbar_wait(&bars->acc_full[ap.acc], ap.phase, bars, pp.err)) return false;
         tc_fence_after();
         const int row = m_tile * kBlockM + row_in_tile;

@@ -80,14 +80,19 @@ def _check_topk_rows(tok, logp, logits, k):
     return tolerated
 
 
-@pytest.mark.parametrize("impl", [0, 1])
+# impl 0: tensor cores, nodes as columns of the MMA for up to 128 rows (the weight-stream form); 1: CUDA-core
+# debug GEMM; 2: tensor cores with one thread per node row at every size
+@pytest.mark.parametrize("impl", [0, 1, 2])
 @pytest.mark.parametrize("rows,V,d,k", [(1, 1024, 256, 4), (12, 1024, 256, 2), (130, 1000, 128, 8),
-                                        (40, 8000, 512, 6), (5, 64, 64, 8), (3, 40, 64, 1)])
+                                        (40, 8000, 512, 6), (5, 64, 64, 8), (3, 40, 64, 1), (16, 32000, 256, 6),
+                                        (96, 20040, 192, 3), (128, 5000, 64, 5), (33, 1000, 200, 8), (64, 129, 72, 7)])
 def test_head_topk_matches_oracle(B, impl, rows, V, d, k):
     cfg = small_cfg(d_base=d, d_inner=d, V=V, topk=(2, 2), seed=rows * 7 + k)
     sw, ow, gw = _setup(cfg)
     h = B.spec_create(gw)
-    B.spec_set_option(h, B.SPEC_OPT_GEMM_IMPL, impl)
+    B.spec_set_option(h, B.SPEC_OPT_GEMM_IMPL, impl & 1)
+    if impl == 2:
+        B.spec_set_option(h, B.SPEC_OPT_HEAD_SWAP_MAX_ROWS, 0)
     S = _states(rows, d, 4)
     tok, logp, ws = B.spec_head_topk(h, 0, S.cuda(), k)
     assert B.spec_poll_error(ws) == 0
@@ -97,9 +102,11 @@ def test_head_topk_matches_oracle(B, impl, rows, V, d, k):
     B.spec_destroy(h)
 
 
-def test_head_topk_exact_ties_prefer_lower_token_id(B):
+@pytest.mark.parametrize("swapped", [False, True])
+def test_head_topk_exact_ties_prefer_lower_token_id(B, swapped):
     """Duplicate output rows give exactly equal logits: the lower token id must come first,
-    also when the two copies sit in different vocabulary tiles."""
+    also when the two copies sit in different vocabulary tiles (and, in the weight-stream form, in
+    different segments of one tile)."""
     cfg = small_cfg(d_base=64, d_inner=64, V=1024, topk=(2, 2), seed=21)
     sw = synth.make_weights(cfg)
     for l in range(cfg.n):
@@ -107,7 +114,8 @@ def test_head_topk_exact_ties_prefer_lower_token_id(B):
         sw.head[l][4] = sw.head[l][3]
     ow, gw = to_oracle_weights(sw), weights_to_cuda(sw)
     h = B.spec_create(gw)
-    B.spec_set_option(h, B.SPEC_OPT_HEAD_BLOCK_N, 32)
+    if not swapped:
+        B.spec_set_option(h, B.SPEC_OPT_HEAD_BLOCK_N, 32)
     # a state aligned with row 3 makes tokens 3, 4 and 700 the tied maximum
     S = (sw.head[0][3].to(torch.float32) * 40).to(torch.bfloat16)[None].contiguous()
     tok, logp, _ = B.spec_head_topk(h, 0, S.cuda(), 4)
