@@ -137,7 +137,8 @@ int spec_draft(spec_handle_t h, const void *ctx_state, const int32_t *last_tok, 
  *   m[b,k]        = number of leading j < n with cand_tok[b,k,j] == g[b,k,j]
  *   best_cand[b]  = lowest k attaining max_k m[b,k];  accept_len[b] = m[b,best];
  *   next_tok[b]   = g[b,best,accept_len[b]]
- *   cand_tok      dev int32 [B, K, n];  base_logits dev [B, K, n+1, V] of logits_dtype
+ *   cand_tok      dev int32 [B, K, n];  base_logits dev [B, K, n+1, V] of logits_dtype (read through the
+ *                 non-coherent path: whatever produces it must precede this call on the stream)
  *   accept_len, best_cand, next_tok  dev int32 [B] (out)
  *   workspace     dev, 256-byte aligned, >= spec_verify_workspace_bytes(...); on return it
  *                 holds the error word (offset 0) and g as int32 [B,K,n+1] at offset 256.

@@ -89,7 +89,7 @@ constexpr int kStreamUnroll = 8;
 template <bool kBf16>
 __global__ void __launch_bounds__(kArgmaxThreads, 4)
 verify_stream_kernel(const uint4 *__restrict__ logits, long long total_vec, int vpr, int vec_per_warp, int slots,
-                     float *__restrict__ pval, int32_t *__restrict__ pidx) {
+                     float *pval, int32_t *pidx) {
     griddep_launch();
     griddep_wait();
     constexpr int kEpv = kBf16 ? 8 : 4;
@@ -163,12 +163,15 @@ verify_argmax_kernel(const void *__restrict__ logits, int rows, int V, int chunk
     }
 }
 
+// (Everything an earlier kernel of the stream wrote - the partials, the candidates, the match lengths and the
+// indices spec_next_ctx consumes - is read with ld.global.cg, never through the non-coherent path: these
+// kernels start early under programmatic dependent launch and the same addresses are rewritten call after call.
+// base_logits itself is streamed with ld.global.nc: it must be complete before the call is enqueued behind
+// its producer on the stream, which stream order guarantees.)
 __global__ void __launch_bounds__(128)
-verify_accept_kernel(const int32_t *__restrict__ cand_tok, const float *__restrict__ pval,
-                     const int32_t *__restrict__ pidx, int K, int n, int slots, int vpr, int vec_per_warp,
-                     int32_t *g_out, int g_in_smem,
-                     int32_t *__restrict__ accept_len, int32_t *__restrict__ best_cand,
-                     int32_t *__restrict__ next_tok, int32_t *err) {
+verify_accept_kernel(const int32_t *cand_tok, const float *pval, const int32_t *pidx, int K, int n, int slots, int vpr,
+                     int vec_per_warp, int32_t *g_out, int g_in_smem, int32_t *accept_len, int32_t *best_cand,
+                     int32_t *next_tok, int32_t *err) {
     // The sequence's arg-max table is re-read by other threads for the prefix match: from shared memory
     // when it fits the default 48 KB, otherwise from the copy in g_out this CTA has just written (global
     // writes of a CTA are visible to its own threads after the barrier).
@@ -191,10 +194,10 @@ verify_accept_kernel(const int32_t *__restrict__ cand_tok, const float *__restri
         float best = -INFINITY;
         int arg = 0;   // a row without any value above -inf (all NaN) yields 0
         for (int c = 0; c < chunks; ++c) {
-            const float v = pval[u0 + c];
+            const float v = __ldcg(pval + u0 + c);
             if (v > best) {   // chunks ascend, so the first maximum wins
                 best = v;
-                arg = pidx[u0 + c];
+                arg = __ldcg(pidx + u0 + c);
             }
         }
         if (g_in_smem) g_s[r] = arg;
@@ -206,7 +209,7 @@ verify_accept_kernel(const int32_t *__restrict__ cand_tok, const float *__restri
         const int32_t *c = cand_tok + ((size_t)b * K + k) * n;
         const int32_t *gk = gtab + k * (n + 1);
         int m = 0;
-        while (m < n && c[m] == gk[m]) ++m;
+        while (m < n && __ldcg(c + m) == gk[m]) ++m;
         // longest prefix first, then the lowest candidate index
         atomicMax(&key_s, ((unsigned)m << 16) | (unsigned)(0xffff - k));
     }
@@ -227,8 +230,8 @@ verify_accept_kernel(const int32_t *__restrict__ cand_tok, const float *__restri
 // B K (n+1) V to sum over candidates of (m + 1) V elements; rows that were not read get g = -1.
 template <bool kBf16>
 __global__ void __launch_bounds__(kArgmaxThreads)
-verify_early_kernel(const uint4 *__restrict__ logits, const int32_t *__restrict__ cand_tok, int n, int vpr,
-                    int32_t *__restrict__ g, int32_t *__restrict__ match_len) {
+verify_early_kernel(const uint4 *__restrict__ logits, const int32_t *cand_tok, int n, int vpr, int32_t *g,
+                    int32_t *match_len) {
     __shared__ float s_val[kWarpsPerBlock];
     __shared__ int s_idx[kWarpsPerBlock];
     __shared__ int s_arg;
@@ -277,7 +280,7 @@ verify_early_kernel(const uint4 *__restrict__ logits, const int32_t *__restrict_
         }
         __syncthreads();
         const int arg = s_arg;
-        if (j < n && cand_tok[(size_t)c * n + j] != arg) {   // uniform over the CTA
+        if (j < n && __ldcg(cand_tok + (size_t)c * n + j) != arg) {   // uniform over the CTA
             m = j;
             break;
         }
@@ -288,9 +291,8 @@ verify_early_kernel(const uint4 *__restrict__ logits, const int32_t *__restrict_
 
 // One CTA per sequence: the candidate with the longest match (lowest index among equals) and its bonus token.
 __global__ void __launch_bounds__(128)
-verify_accept_early_kernel(const int32_t *__restrict__ g, const int32_t *__restrict__ match_len, int K, int n,
-                           int32_t *__restrict__ accept_len, int32_t *__restrict__ best_cand,
-                           int32_t *__restrict__ next_tok, int32_t *err) {
+verify_accept_early_kernel(const int32_t *g, const int32_t *match_len, int K, int n, int32_t *accept_len,
+                           int32_t *best_cand, int32_t *next_tok, int32_t *err) {
     __shared__ unsigned int key_s;
     griddep_launch();
     griddep_wait();
@@ -301,13 +303,13 @@ verify_accept_early_kernel(const int32_t *__restrict__ g, const int32_t *__restr
     }
     __syncthreads();
     for (int k = threadIdx.x; k < K; k += blockDim.x)
-        atomicMax(&key_s, ((unsigned)match_len[(size_t)b * K + k] << 16) | (unsigned)(0xffff - k));
+        atomicMax(&key_s, ((unsigned)__ldcg(match_len + (size_t)b * K + k) << 16) | (unsigned)(0xffff - k));
     __syncthreads();
     if (threadIdx.x == 0) {
         const int m = (int)(key_s >> 16), k = 0xffff - (int)(key_s & 0xffffu);
         accept_len[b] = m;
         best_cand[b] = k;
-        next_tok[b] = g[((size_t)b * K + k) * (n + 1) + m];
+        next_tok[b] = __ldcg(g + ((size_t)b * K + k) * (n + 1) + m);
     }
 }
 
@@ -430,13 +432,12 @@ namespace {
 // One CTA per sequence copies base_state[b, best_cand[b], accept_len[b], :] to ctx_state[b, :].  The two
 // indices come from the verify kernels earlier in the stream, hence the dependency wait before they are read.
 __global__ void __launch_bounds__(128)
-next_ctx_kernel(const uint16_t *__restrict__ base_state, const int32_t *__restrict__ best_cand,
-                const int32_t *__restrict__ accept_len, int K, int n, int d, int vec_ok,
-                uint16_t *__restrict__ ctx_state, int32_t *err) {
+next_ctx_kernel(const uint16_t *__restrict__ base_state, const int32_t *best_cand, const int32_t *accept_len, int K,
+                int n, int d, int vec_ok, uint16_t *__restrict__ ctx_state, int32_t *err) {
     griddep_launch();
     griddep_wait();
     const int b = blockIdx.x;
-    const int k = best_cand[b], m = accept_len[b];
+    const int k = __ldcg(best_cand + b), m = __ldcg(accept_len + b);
     uint16_t *dst = ctx_state + (size_t)b * d;
     if (k < 0 || k >= K || m < 0 || m > n) {   // never read outside the tensor: the row becomes zero
         if (threadIdx.x == 0) report_error(err, SPEC_ERR_INDEX_RANGE);
