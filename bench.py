@@ -178,6 +178,8 @@ def run_only(args, cfg, peaks, dev):
             B.spec_set_option(h, B.SPEC_OPT_HEAD_BLOCK_N, args.block_n)
         if args.swap_max_rows is not None:
             B.spec_set_option(h, B.SPEC_OPT_HEAD_SWAP_MAX_ROWS, args.swap_max_rows)
+        if args.producers:
+            B.spec_set_option(h, B.SPEC_OPT_GEMM_PRODUCERS, args.producers)
         g = torch.Generator(device=dev).manual_seed(5)
         S = (torch.randn(rows, cfg.d_inner, generator=g, device=dev) * 0.5).to(torch.bfloat16)
         tok = torch.empty((rows, k), dtype=torch.int32, device=dev)
@@ -226,6 +228,7 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--swap-max-rows", type=int, default=None,
                     help="--only head*: levels of at most this many rows use the weight-stream form (0: never)")
+    ap.add_argument("--producers", type=int, default=0, help="--only head*: TMA-issuing threads per CTA (1 or 2)")
     ap.add_argument("--vocab", type=int, default=None, help="--only head*: vocabulary size instead of the workload's")
     ap.add_argument("--topk", type=int, default=None, help="--only head*: branching factor (default: the last level's)")
     ap.add_argument("--only", default=None, choices=["head", "head_gemm", "verify"],

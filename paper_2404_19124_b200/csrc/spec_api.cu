@@ -414,6 +414,10 @@ int spec_set_option(spec_handle_t h, int option, int value) {
             if (value < 0 || value > (1 << 24)) return SPEC_ERR_INVALID_ARG;
             h->fp8_max_rows = value;
             return SPEC_OK;
+        case SPEC_OPT_GEMM_PRODUCERS:
+            if (value != 1 && value != 2) return SPEC_ERR_INVALID_ARG;
+            set_gemm_producers(value);
+            return SPEC_OK;
         case SPEC_OPT_HEAD_SWAP_MAX_ROWS:
             if (value < 0 || value > 128) return SPEC_ERR_INVALID_ARG;
             h->swap_max_rows = value;

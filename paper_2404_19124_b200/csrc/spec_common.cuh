@@ -115,6 +115,7 @@ struct GemmEpilogue {
 // Mode 3 bookkeeping, the same on the host (workspace sizing, merge) and in the launch.
 int swapped_head_segs(int nodes);
 int swapped_head_parts(int nodes, int vocab_rows);
+void set_gemm_producers(int n);   // process-wide: 1 or 2 TMA-issuing threads per CTA
 int choose_block_n(int M, int N, int num_sm, bool tensor_bound_pref);
 int launch_gemm_tc(const void *A, const void *B, int M, int N, int Kd, int block_n, const GemmEpilogue &epi,
                    int32_t *err, cudaStream_t st);

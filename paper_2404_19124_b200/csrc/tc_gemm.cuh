@@ -2,9 +2,9 @@
 //     C[M, N] = A[M, Kd] * B[N, Kd]^T,  bf16 operands (row-major = K-major for both), fp32 in TMEM,
 // used by the GEMM kernel (gemm_tcgen05.cu).
 //
-// A CTA has 192 threads in three roles that meet only through mbarriers:
-//   warp 0      TMA producer: 128-byte-swizzled [128 x 64] A boxes and [block_n x 64] B boxes into a
-//               ring of shared-memory slots, completion on "full" barriers
+// A CTA has 224 threads in three roles that meet only through mbarriers:
+//   warps 0, 6  TMA producers (one lane each, alternating ring slots): 128-byte-swizzled [128 x 64] A boxes
+//               and [block_n x 64] B boxes into a ring of shared-memory slots, completion on "full" barriers
 //   warp 1      owns the TMEM allocation; one lane issues tcgen05.mma (M 128, N block_n, K 16) and
 //               commits to the slot's "empty" barrier and, per tile, to "accumulator full"
 //   warps 2-5   epilogue: tcgen05.ld of 32 columns at a time, one thread per accumulator row
@@ -31,7 +31,10 @@ namespace tc {
 constexpr int kBlockM = 128;
 constexpr int kSlabBytes = 128;        // one K block = one 128-byte swizzle span per row: 64 bf16 or 128 fp8 elements
 constexpr int kUmmaBytes = 32;         // K extent of one MMA instruction in bytes: 16 bf16 or 32 fp8 elements
-constexpr int kThreads = 192;
+constexpr int kMaxProducers = 2;       // TMA-issuing threads (lane 0 of warp 0 and, optionally, of warp 6, alternating
+                                       // the ring slots)
+constexpr int kThreads = 224;
+constexpr int kEpilogueFirst = 64;     // first epilogue thread
 constexpr int kEpilogueThreads = 128;  // warps 2-5
 constexpr int kMaxStages = 12;
 constexpr int kABytes = kBlockM * kSlabBytes;
@@ -321,10 +324,12 @@ __device__ __forceinline__ void advance(const Pipe &pp, RingPos &rp) {
 // the preceding grid has completed, or the grid-wide barrier behind which they are written has
 // opened) and the state operand of those slots follows.  A CTA without a tile in the job neither
 // loads nor waits.  `issued` counts slots filled since the kernel started (for the abort path).
+// Producer `me` of `n_prod` walks every slot like the others and fills the slots whose running number
+// `issued` (counted over all jobs of the launch) is congruent to `me`.
 template <typename DepWait>
 __device__ __forceinline__ bool produce_job(const Pipe &pp, const GemmJob &j, const CUtensorMap *tmap_a,
                                             const CUtensorMap *tmap_a_short, const CUtensorMap *tmap_b, RingPos &rp,
-                                            int &issued, DepWait dep_wait) {
+                                            int &issued, int me, int n_prod, DepWait dep_wait) {
     const int ke = slab_elems(j);
     const uint32_t b_bytes = (uint32_t)j.block_n * kSlabBytes;
     const TileWalk w = walk_of(j);
@@ -338,11 +343,13 @@ __device__ __forceinline__ bool produce_job(const Pipe &pp, const GemmJob &j, co
         n_pre = min(pp.stages, t0.kb1 - t0.kb0);
         RingPos q = rp;
         for (int i = 0; i < n_pre; ++i) {
-            if (!mbar_wait(&bars->empty[q.stage], q.phase ^ 1u, bars, pp.err)) return false;
-            uint8_t *sa = pp.tiles + (size_t)q.stage * pp.slot_bytes;
-            mbar_arrive_expect_tx(&bars->full[q.stage], tx);
-            if (j.w_is_a) tma_load_2d(sa, ma, (t0.kb0 + i) * ke, t0.a_row, &bars->full[q.stage]);
-            else tma_load_2d(sa + kABytes, tmap_b, (t0.kb0 + i) * ke, t0.b_row, &bars->full[q.stage]);
+            if ((issued + i) % n_prod == me) {
+                if (!mbar_wait(&bars->empty[q.stage], q.phase ^ 1u, bars, pp.err)) return false;
+                uint8_t *sa = pp.tiles + (size_t)q.stage * pp.slot_bytes;
+                mbar_arrive_expect_tx(&bars->full[q.stage], tx);
+                if (j.w_is_a) tma_load_2d(sa, ma, (t0.kb0 + i) * ke, t0.a_row, &bars->full[q.stage]);
+                else tma_load_2d(sa + kABytes, tmap_b, (t0.kb0 + i) * ke, t0.b_row, &bars->full[q.stage]);
+            }
             advance(pp, q);
         }
     }
@@ -356,12 +363,14 @@ __device__ __forceinline__ bool produce_job(const Pipe &pp, const GemmJob &j, co
             uint8_t *sa = pp.tiles + (size_t)rp.stage * pp.slot_bytes;
             uint8_t *sb = sa + kABytes;
             const bool prefetched = done < n_pre;   // the weights of this slot are already on their way
-            if (!prefetched) {
-                if (!mbar_wait(&bars->empty[rp.stage], rp.phase ^ 1u, bars, pp.err)) return false;
-                mbar_arrive_expect_tx(&bars->full[rp.stage], tx);
+            if (issued % n_prod == me) {
+                if (!prefetched) {
+                    if (!mbar_wait(&bars->empty[rp.stage], rp.phase ^ 1u, bars, pp.err)) return false;
+                    mbar_arrive_expect_tx(&bars->full[rp.stage], tx);
+                }
+                if (!prefetched || !j.w_is_a) tma_load_2d(sa, ma, kb * ke, t.a_row, &bars->full[rp.stage]);
+                if (!prefetched || j.w_is_a) tma_load_2d(sb, tmap_b, kb * ke, t.b_row, &bars->full[rp.stage]);
             }
-            if (!prefetched || !j.w_is_a) tma_load_2d(sa, ma, kb * ke, t.a_row, &bars->full[rp.stage]);
-            if (!prefetched || j.w_is_a) tma_load_2d(sb, tmap_b, kb * ke, t.b_row, &bars->full[rp.stage]);
             ++done;
             ++issued;
             advance(pp, rp);
@@ -370,7 +379,8 @@ __device__ __forceinline__ bool produce_job(const Pipe &pp, const GemmJob &j, co
     return true;
 }
 
-// After a failed wait: let the copies already in flight land before the CTA's shared memory is released.
+// After a failed wait: let the copies already in flight land before the CTA's shared memory is released
+// (every producer waits for all recent slots, its own and the others').
 __device__ __forceinline__ void producer_drain(const Pipe &pp, RingPos rp, int issued) {
     const int pending = issued < pp.stages ? issued : pp.stages;
     for (int i = 0; i < pending; ++i) {
@@ -732,7 +742,7 @@ __device__ __forceinline__ bool epilogue_job_swapped(const Pipe &pp, const GemmJ
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int quarter = warp & 3;                    // TMEM lane quarter this warp may read
     const int vrow = quarter * 32 + lane;            // vocabulary row of the tile held by this thread's TMEM lane
-    const int u = (int)threadIdx.x - (kThreads - kEpilogueThreads);
+    const int u = (int)threadIdx.x - kEpilogueFirst;
     const int nodes = j.N, P = j.epi.segs, len = kBlockM / P;
     const int node = u / P, seg = u - node * P;
     const bool scans = node < nodes;
