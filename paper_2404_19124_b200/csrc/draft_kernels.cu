@@ -104,18 +104,21 @@ struct MergeMixArgs {
     MixArgs mix;       // level l + 1 (tok and parent_div unused: the tokens come from the merge)
 };
 
-__global__ void __launch_bounds__(kRowThreads, 1) merge_mix_kernel(MergeMixArgs a) {
+// At most 128 registers: like the other row kernels its CTAs must fit beside a resident GEMM CTA, or they could
+// not start (and wait, set up) before that kernel ends.
+constexpr int kFusedBatch = 2;
+__global__ void __launch_bounds__(kRowThreads, 2) merge_mix_kernel(MergeMixArgs a) {
     __shared__ Scratch sc;
-    __shared__ float red_a[kRowThreads / 32 * 4], red_b[kRowThreads / 32 * 4];
+    __shared__ float red_a[kRowThreads / 32 * kFusedBatch], red_b[kRowThreads / 32 * kFusedBatch];
     griddep_launch();
     griddep_wait();
     const int r = blockIdx.x, tid = threadIdx.x;
     merge_expand_row<kRowThreads, BlockSync>(a.merge, r, tid, &sc);
     // sc.out_id[0 .. topk) now hold the children's tokens (valid for the whole CTA after merge_select's last barrier)
     if (a.mix.d <= 8 * kRowThreads)
-        mix_children<kRowThreads, 1, BlockSync>(a.mix, r, r * a.merge.topk, a.merge.topk, sc.out_id, red_a, red_b, tid);
+        mix_children<kRowThreads, 1, kFusedBatch, BlockSync>(a.mix, r, r * a.merge.topk, a.merge.topk, sc.out_id, red_a, red_b, tid);
     else
-        mix_children<kRowThreads, 2, BlockSync>(a.mix, r, r * a.merge.topk, a.merge.topk, sc.out_id, red_a, red_b, tid);
+        mix_children<kRowThreads, 2, kFusedBatch, BlockSync>(a.mix, r, r * a.merge.topk, a.merge.topk, sc.out_id, red_a, red_b, tid);
 }
 
 // Vocabulary-parallel head: one warp per row folds the n_ranks raw lists (see launch_merge_shards).

@@ -387,11 +387,10 @@ __device__ __forceinline__ void merge_expand_row(const MergeArgs &g, int r, int 
 // row of child 0 in the next level.  The projected parent state (sum of the split-K partials, added in
 // ascending order) and the LayerNorm parameters are loaded once; per trip the embedding rows of the batch
 // are requested together and the two LayerNorm reductions are done for the whole batch with one barrier
-// each (red_a / red_b: kThreads / 32 x kBatch floats each).  d <= 8 * kThreads * kIters, d % 8 == 0.
-template <int kThreads, int kIters, typename Sync>
+// each (red_a / red_b: kThreads / 32 x kBatch floats each; kBatch children per trip).  d <= 8 * kThreads * kIters, d % 8 == 0.
+template <int kThreads, int kIters, int kBatch, typename Sync>
 __device__ __forceinline__ void mix_children(const MixArgs &m, int parent, int first_child, int n_child, const int *tok,
                                              float *red_a, float *red_b, int tid) {
-    constexpr int kBatch = 4;
     constexpr int kWarps = kThreads / 32;
     const int d = m.d, lane = tid & 31, warp = tid >> 5;
     float pv[kIters][8], gv[kIters][8], bv[kIters][8];
