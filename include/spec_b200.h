@@ -59,11 +59,12 @@ enum spec_option {
                                   one is attached (default 128, the levels bound by the weight
                                   stream; 0 = never).  Larger values put tensor-bound levels on
                                   the e4m3 path too, which pays from about 768 nodes on        */
-    SPEC_OPT_HEAD_SWAP_MAX_ROWS = 5, /* levels with at most this many nodes (0 .. 128, default 128) run
-                                  the head GEMM with the weight matrix on the 128-row side of the
-                                  MMA and the nodes as columns, so the tensor work follows the
-                                  number of nodes and the launch is a pure weight stream; 0 = never.
-                                  Ignored while SPEC_OPT_HEAD_BLOCK_N forces a tile width.     */
+    SPEC_OPT_HEAD_SWAP_MAX_ROWS = 5, /* levels with at most this many nodes (0 .. 128) run the head GEMM
+                                  with the weight matrix on the 128-row side of the MMA and the nodes
+                                  as columns, so the tensor work follows the number of nodes; 0 = never;
+                                  -1 (default) = automatic: up to 8 nodes, or up to 32 when the
+                                  vocabulary gives every CTA at least four 128-row tiles.  Ignored
+                                  while SPEC_OPT_HEAD_BLOCK_N forces a tile width.              */
     SPEC_OPT_GEMM_PRODUCERS = 6  /* 1 or 2 (default) threads per CTA issue the TMA copies of the GEMM
                                   kernels; process-wide, not per handle                        */
 };

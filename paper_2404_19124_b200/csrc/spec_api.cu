@@ -76,8 +76,15 @@ int head_block_n_for(const spec_handle_s *h, int rows) {
 }
 
 // Levels of few nodes run the head with the weights on the 128-row side of the MMA (epilogue mode 3).
+// Which levels: set explicitly, or by what measured faster inside whole drafts.  The swapped form costs fewer
+// TMA requests and MMA cycles per weight byte but ends every CTA with a longer epilogue (transposition, scan,
+// combination of the segment lists), which only a long weight stream pays back: up to 8 nodes at any
+// vocabulary, up to 32 nodes when every CTA streams at least four 128-row tiles (V = 128256: 121 against
+// 137 us at 16 nodes); at 16 nodes and V = 32000 the one-thread-per-node form is 2-3 us per level faster.
 bool head_swapped_for(const spec_handle_s *h, int rows) {
-    return h->gemm_impl == 0 && h->head_block_n == 0 && rows <= h->swap_max_rows && rows <= 128;
+    if (h->gemm_impl != 0 || h->head_block_n != 0 || rows > 128) return false;
+    if (h->swap_max_rows >= 0) return rows <= h->swap_max_rows;
+    return rows <= 8 || (rows <= 32 && h->head_rows >= 4 * 128 * num_sms());
 }
 
 // Partial lists per row that the head of `rows` nodes leaves for the merge, and its tile width.
@@ -367,7 +374,7 @@ int spec_create(spec_handle_t *out, const spec_weights_t *w) {
     h->proj_block_n = 0;
     h->profile = 0;
     h->fp8_max_rows = 128;
-    h->swap_max_rows = 128;
+    h->swap_max_rows = -1;
     h->vp_rank = 0;
     h->vp_ranks = 1;
     h->vocab_offset = 0;
@@ -419,7 +426,7 @@ int spec_set_option(spec_handle_t h, int option, int value) {
             set_gemm_producers(value);
             return SPEC_OK;
         case SPEC_OPT_HEAD_SWAP_MAX_ROWS:
-            if (value < 0 || value > 128) return SPEC_ERR_INVALID_ARG;
+            if (value < -1 || value > 128) return SPEC_ERR_INVALID_ARG;
             h->swap_max_rows = value;
             return SPEC_OK;
         default:

@@ -91,8 +91,7 @@ def test_head_topk_matches_oracle(B, impl, rows, V, d, k):
     sw, ow, gw = _setup(cfg)
     h = B.spec_create(gw)
     B.spec_set_option(h, B.SPEC_OPT_GEMM_IMPL, impl & 1)
-    if impl == 2:
-        B.spec_set_option(h, B.SPEC_OPT_HEAD_SWAP_MAX_ROWS, 0)
+    B.spec_set_option(h, B.SPEC_OPT_HEAD_SWAP_MAX_ROWS, 0 if impl == 2 else 128)
     S = _states(rows, d, 4)
     tok, logp, ws = B.spec_head_topk(h, 0, S.cuda(), k)
     assert B.spec_poll_error(ws) == 0
@@ -114,7 +113,9 @@ def test_head_topk_exact_ties_prefer_lower_token_id(B, swapped):
         sw.head[l][4] = sw.head[l][3]
     ow, gw = to_oracle_weights(sw), weights_to_cuda(sw)
     h = B.spec_create(gw)
-    if not swapped:
+    if swapped:
+        B.spec_set_option(h, B.SPEC_OPT_HEAD_SWAP_MAX_ROWS, 128)
+    else:
         B.spec_set_option(h, B.SPEC_OPT_HEAD_BLOCK_N, 32)
     # a state aligned with row 3 makes tokens 3, 4 and 700 the tied maximum
     S = (sw.head[0][3].to(torch.float32) * 40).to(torch.bfloat16)[None].contiguous()
@@ -126,7 +127,8 @@ def test_head_topk_exact_ties_prefer_lower_token_id(B, swapped):
     B.spec_destroy(h)
 
 
-def _draft_and_check(B, cfg, seqs=None, impl=0, check_levels=False, tie_weights=False, fp8=False, fp8_rows=None):
+def _draft_and_check(B, cfg, seqs=None, impl=0, check_levels=False, tie_weights=False, fp8=False, fp8_rows=None,
+                     swap=None):
     """Runs spec_draft at the config's full batch and compares the sequences in `seqs`
     (default: all) with the oracle, one sequence at a time (sequences are independent).
     tie_weights: every head after the first aliases the second head's tensors (the weight-tied
@@ -145,6 +147,8 @@ def _draft_and_check(B, cfg, seqs=None, impl=0, check_levels=False, tie_weights=
     ctx, tok = synth.make_draft_inputs(cfg)
     h = B.spec_create(gw)
     B.spec_set_option(h, B.SPEC_OPT_GEMM_IMPL, impl)
+    if swap is not None:   # levels of up to `swap` nodes run the head with the nodes as MMA columns (0: none)
+        B.spec_set_option(h, B.SPEC_OPT_HEAD_SWAP_MAX_ROWS, swap)
     if fp8:      # levels of up to 128 nodes multiply in e4m3 and re-score a short list exactly
         B.spec_attach_fp8_heads(h)
         if fp8_rows is not None:   # also levels with more than the default 128 nodes
@@ -202,9 +206,10 @@ def test_draft_tiny_config(B, impl):
 @pytest.mark.parametrize("topk,K,Bn,V,d_base,d", [((3, 2, 2), 5, 2, 1000, 72, 64), ((1, 1, 1), 1, 3, 512, 64, 64),
                                                    ((8, 8), 64, 2, 2048, 128, 192), ((2, 2, 2, 2, 2), 7, 5, 640, 64, 128),
                                                    ((4, 3), 12, 150, 512, 64, 64)])
-def test_draft_odd_shapes(B, topk, K, Bn, V, d_base, d):
+@pytest.mark.parametrize("swap", [0, 128])
+def test_draft_odd_shapes(B, topk, K, Bn, V, d_base, d, swap):
     cfg = small_cfg(d_base=d_base, d_inner=d, V=V, topk=topk, K=K, B=Bn, seed=len(topk) + Bn)
-    chk = _draft_and_check(B, cfg, check_levels=True)
+    chk = _draft_and_check(B, cfg, check_levels=True, swap=swap)
     assert chk.tolerated <= max(1, Bn // 5)
 
 
@@ -222,12 +227,23 @@ def test_draft_weight_tied_heads(B):
     assert chk.tolerated <= 1
 
 
-def test_draft_single_candidate_at_production_width(B):
-    """k = 1 (Sec. 4.2 / Sec. 5: the setting the paper recommends under load): topk = 1 at every head,
-    one candidate per sequence, at the Llama2-7B-shaped widths."""
+@pytest.mark.parametrize("name,Bn", [("llama2-7b", 1), ("llama2-7b", 16), ("llama2-7b", 64), ("llama2-13b", 1),
+                                     ("llama2-13b", 16), ("llama2-13b", 64)])
+def test_draft_single_candidate_at_production_width(B, name, Bn):
+    """k = 1 (Sec. 4.2 / Sec. 5: the setting the paper recommends under load): topk = 1 at every head, one
+    candidate per sequence, at the Llama2-7B- and 13B-shaped widths.  This is the chain of eight launches
+    (the merge of a level also writes the one child's state): the candidate is the greedy chain."""
     import dataclasses
-    cfg = dataclasses.replace(synth.CONFIGS["llama2-7b"], topk=(1, 1, 1), K=1, B=4)
-    chk = _draft_and_check(B, cfg)
+    cfg = dataclasses.replace(synth.CONFIGS[name], topk=(1, 1, 1), K=1, B=Bn)
+    chk = _draft_and_check(B, cfg, seqs=range(0, Bn, max(1, Bn // 4)), check_levels=False)
+    assert chk.tolerated <= 1
+
+
+@pytest.mark.parametrize("topk,K", [((2, 2, 2), 5), ((2, 1, 2, 1), 3), ((1, 2, 1), 2)])
+def test_draft_one_or_two_children_per_node(B, topk, K):
+    """Branching factors of one and two: the merge of a level writes the children's states in the same launch."""
+    cfg = small_cfg(d_base=96, d_inner=160, V=3000, topk=topk, K=K, B=5, seed=11 + len(topk))
+    chk = _draft_and_check(B, cfg, check_levels=True)
     assert chk.tolerated <= 1
 
 
@@ -309,9 +325,10 @@ def _report_tolerated(record_property, name, chk, checked):
     record_property("checked", checked)
 
 
-def test_draft_llama2_7b_shape(B, record_property):
+@pytest.mark.parametrize("swap", [None, 128])
+def test_draft_llama2_7b_shape(B, record_property, swap):
     cfg = synth.CONFIGS["llama2-7b"]
-    chk = _draft_and_check(B, cfg)
+    chk = _draft_and_check(B, cfg, swap=swap)
     _report_tolerated(record_property, cfg.name, chk, cfg.B)
     assert chk.exact + chk.tolerated == cfg.B
     # near-ties after a bf16 rounding flip (the synthetic heads give nearly flat distributions, so leaf scores
