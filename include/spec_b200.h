@@ -134,6 +134,27 @@ int spec_draft_layout(spec_handle_t h, int B, const int32_t *topk, int K, spec_d
 int spec_draft(spec_handle_t h, const void *ctx_state, const int32_t *last_tok, int B, const int32_t *topk, int K,
                int32_t *cand_tok, float *cand_logp, void *workspace, size_t workspace_bytes, void *cuda_stream);
 
+/* ---- how many candidates to draft (Sec. 4.2 and Sec. 5: several candidates per sequence pay at batch size 1
+ * - the paper quotes k = 5 there - a single candidate, k = 1, is the better setting under load, and beyond some
+ * batch size speculation is switched off altogether because the base model's forward over B * k * (n + 1)
+ * tokens becomes compute-bound).  The paper gives the shape of that rule, not its numbers, which depend on the
+ * base model and the GPU: they are the caller's, as a table sorted by ascending batch size.
+ *   rules     host, n_rules entries with strictly ascending max_batch; entry i applies to
+ *             B <= rules[i].max_batch (and B > rules[i-1].max_batch).  K = 0 in an entry means "do not
+ *             speculate"; otherwise topk[0 .. n_heads) are the branching factors to draft with
+ *             (1 <= topk[l] <= SPEC_MAX_TOPK, K <= prod topk <= SPEC_MAX_LEAVES).
+ *   K_out     host: receives the K of the first entry that covers B, 0 when B is larger than every max_batch
+ *   topk_out  host int32 [n_heads], may be NULL: receives that entry's branching factors (zeros when K = 0)
+ * Host-only: touches no device and no stream.  SPEC_ERR_INVALID_ARG for a malformed table.
+ * With K = 1 and topk = 1 everywhere spec_draft runs its shortest launch chain: every head has B rows, a
+ * level's top-k is an arg-max and its merge also writes the one child's state. */
+typedef struct {
+    int32_t max_batch;
+    int32_t K;
+    int32_t topk[SPEC_MAX_HEADS];
+} spec_k_rule_t;
+int spec_choose_k(int B, int n_heads, const spec_k_rule_t *rules, int n_rules, int32_t *K_out, int32_t *topk_out);
+
 /* ---- verify (Sec. 1: accept the speculated tokens that match the base model's outputs;
  * Sec. 3.1: score all candidates, keep the best; Sec. 5: at most n + 1 tokens per step) --
  *   g[b,k,j]      = first index of the maximum of base_logits[b,k,j,:] (NaN never wins)

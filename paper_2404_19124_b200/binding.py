@@ -29,7 +29,7 @@ EXPORTS = [
     "spec_draft_workspace_bytes", "spec_draft_layout", "spec_draft", "spec_verify_workspace_bytes", "spec_verify",
     "spec_profile_read", "spec_poll_error", "spec_head_workspace_bytes", "spec_head_logits", "spec_head_topk",
     "spec_verify_static", "spec_verify_early", "spec_quantize_head", "spec_set_head_fp8",
-    "spec_head_partials", "spec_next_ctx",
+    "spec_head_partials", "spec_next_ctx", "spec_choose_k",
     "spec_set_vocab_shard", "spec_draft_vp_exchange", "spec_draft_vp_local", "spec_draft_vp_merge",
 ]
 
@@ -77,6 +77,7 @@ _lib.spec_verify_workspace_bytes.restype = C.c_size_t
 _lib.spec_verify_workspace_bytes.argtypes = [C.c_int] * 5
 _lib.spec_verify.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_int, C.c_int, C.c_int,
                              C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]
+_lib.spec_choose_k.argtypes = [C.c_int, C.c_int, C.c_void_p, C.c_int, C.c_void_p, C.c_void_p]
 _lib.spec_verify_static.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_int, C.c_int, C.c_int,
                                     C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
 _lib.spec_verify_early.argtypes = _lib.spec_verify.argtypes
@@ -285,6 +286,24 @@ def spec_draft_vp_merge(h: SpecHandle, level: int, B: int, topk: Sequence[int], 
 
 def spec_verify_workspace_bytes(B: int, K: int, n: int, V: int, logits_dtype: int) -> int:
     return int(_lib.spec_verify_workspace_bytes(B, K, n, V, logits_dtype))
+
+
+class SpecKRuleC(C.Structure):
+    _fields_ = [("max_batch", C.c_int32), ("K", C.c_int32), ("topk", C.c_int32 * MAX_HEADS)]
+
+
+def spec_choose_k(B: int, n_heads: int, rules: Sequence[Tuple[int, int, Sequence[int]]]) -> Tuple[int, Tuple[int, ...]]:
+    """rules: (max_batch, K, topk) entries by ascending max_batch; returns (K, topk) for a batch of B sequences,
+    (0, ()) when speculation is off at that batch size.  Host-only."""
+    arr = (SpecKRuleC * len(rules))()
+    for i, (mb, K, topk) in enumerate(rules):
+        arr[i].max_batch, arr[i].K = int(mb), int(K)
+        for l, t in enumerate(topk):
+            arr[i].topk[l] = int(t)
+    K_out = C.c_int32(0)
+    tk = (C.c_int32 * MAX_HEADS)()
+    _check(_lib.spec_choose_k(int(B), int(n_heads), arr, len(rules), C.byref(K_out), tk), "spec_choose_k")
+    return int(K_out.value), (tuple(int(tk[l]) for l in range(n_heads)) if K_out.value > 0 else ())
 
 
 def spec_verify(cand_tok: torch.Tensor, base_logits: torch.Tensor, accept_len: Optional[torch.Tensor] = None,

@@ -618,6 +618,34 @@ int spec_draft(spec_handle_t h, const void *ctx_state, const int32_t *last_tok, 
     return SPEC_OK;
 }
 
+int spec_choose_k(int B, int n_heads, const spec_k_rule_t *rules, int n_rules, int32_t *K_out, int32_t *topk_out) {
+    if (B <= 0 || n_heads < 1 || n_heads > SPEC_MAX_HEADS || !rules || n_rules < 1 || !K_out) return SPEC_ERR_INVALID_ARG;
+    for (int i = 0; i < n_rules; ++i) {
+        const spec_k_rule_t &r = rules[i];
+        if (r.max_batch < 1 || (i > 0 && r.max_batch <= rules[i - 1].max_batch) || r.K < 0) return SPEC_ERR_INVALID_ARG;
+        if (r.K > 0) {
+            long long leaves = 1;
+            for (int l = 0; l < n_heads; ++l) {
+                if (r.topk[l] < 1 || r.topk[l] > SPEC_MAX_TOPK) return SPEC_ERR_INVALID_ARG;
+                leaves *= r.topk[l];
+            }
+            if (leaves > SPEC_MAX_LEAVES || r.K > leaves) return SPEC_ERR_INVALID_ARG;
+        }
+    }
+    *K_out = 0;
+    if (topk_out)
+        for (int l = 0; l < n_heads; ++l) topk_out[l] = 0;
+    for (int i = 0; i < n_rules; ++i) {
+        if (B <= rules[i].max_batch) {
+            *K_out = rules[i].K;
+            if (topk_out && rules[i].K > 0)
+                for (int l = 0; l < n_heads; ++l) topk_out[l] = rules[i].topk[l];
+            break;
+        }
+    }
+    return SPEC_OK;
+}
+
 /* ---- vocabulary-parallel heads ------------------------------------------------------------------ */
 int spec_set_vocab_shard(spec_handle_t h, int rank, int n_ranks, int vocab_offset, int head_rows) {
     if (!h) return SPEC_ERR_INVALID_ARG;

@@ -74,3 +74,28 @@ def test_create_rejects_bad_weights_and_missing_device(binding):
         # the product path refuses to run without a device instead of falling back to anything
         assert binding._lib.spec_create(C.byref(h), C.byref(w)) == binding.SPEC_ERR_NO_DEVICE
         assert not h.value
+
+
+def test_choose_k_follows_the_callers_batch_table(binding):
+    """Sec. 4.2 / Sec. 5: several candidates at batch size 1 (the paper quotes k = 5 with 6/3/2 branching pruned
+    to k, Sec. 4.1), one candidate under load, speculation off beyond a batch size.  The thresholds are the
+    caller's; the call only looks the batch size up.  Runs on the host, no device needed."""
+    rules = [(1, 5, (6, 3, 2)), (8, 2, (2, 1, 1)), (32, 1, (1, 1, 1)), (64, 0, ())]
+    want = {1: (5, (6, 3, 2)), 2: (2, (2, 1, 1)), 8: (2, (2, 1, 1)), 9: (1, (1, 1, 1)), 32: (1, (1, 1, 1)),
+            33: (0, ()), 64: (0, ()), 65: (0, ()), 10 ** 6: (0, ())}
+    for b, w in want.items():
+        assert binding.spec_choose_k(b, 3, rules) == w
+    bad = [
+        [(4, 1, (1, 1, 1)), (4, 0, ())],            # max_batch not strictly ascending
+        [(4, 5, (2, 2, 1))],                        # K beyond the leaves
+        [(4, 1, (1, 0, 1))],                        # a branching factor of zero
+        [(4, 1, (9, 1, 1))],                        # beyond SPEC_MAX_TOPK
+        [(0, 1, (1, 1, 1))],                        # a batch limit below one
+        [(4, -1, (1, 1, 1))],
+    ]
+    for table in bad:
+        with pytest.raises(binding.SpecError) as e:
+            binding.spec_choose_k(2, 3, table)
+        assert e.value.status == binding.SPEC_ERR_INVALID_ARG
+    with pytest.raises(binding.SpecError):
+        binding.spec_choose_k(0, 3, rules)
