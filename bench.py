@@ -116,8 +116,23 @@ def oracle_weights(sw):
         state_weight=sw.state_weight, emb_weight=sw.emb_weight, ln_eps=sw.ln_eps)
 
 
+def workload_config(cfg, world: int, n_rot: int):
+    """The `config` object of the JSON line: the same keys in the GPU arm and in the reference arm."""
+    return {"workload": cfg.name, "B": cfg.B, "K": cfg.K, "n_heads": cfg.n, "topk": list(cfg.topk), "V": cfg.V,
+            "d_base": cfg.d_base, "d_inner": cfg.d_inner, "logits_dtype": "bf16",
+            "l2": f"weights of more than 1 GB per step exceed L2; verify rotates over {n_rot} distinct logits buffers",
+            "parallelism": f"replicas x{world}, sequences independent, no collective"}
+
+
+def logits_rotation(cfg) -> int:
+    """Distinct base_logits buffers a run rotates over (at least 512 MB together, 2 to 8 of them)."""
+    logits_bytes = cfg.B * cfg.K * (cfg.n + 1) * cfg.V * 2
+    return max(2, min(8, (512 << 20) // logits_bytes + 1))
+
+
 def time_oracle(cfg, sw, seqs: int, repeats: int):
-    """Oracle draft + verify on the first `seqs` sequences of the workload; returns seconds per repeat."""
+    """Oracle draft + verify on the first `seqs` sequences of the workload.
+    Returns ([(draft seconds, verify seconds)] per repeat, threads used)."""
     import numpy as np
     import oracle
     from paper_2404_19124_b200 import synth
@@ -130,8 +145,9 @@ def time_oracle(cfg, sw, seqs: int, repeats: int):
     for _ in range(repeats):
         t0 = time.perf_counter()
         ct, _ = oracle.draft(ow, ctx_bits, tok_np, cfg.topk, cfg.K)
+        t1 = time.perf_counter()
         oracle.verify(ct, logits, oracle.BF16)
-        times.append(time.perf_counter() - t0)
+        times.append((t1 - t0, time.perf_counter() - t1))
     return times, oracle.num_threads()
 
 
@@ -140,23 +156,143 @@ def run_reference(args, cfg):
     sw = synth.make_weights(cfg, device="cpu")
     # sequences per step: as many of the batch as keep the whole run to about two minutes of CPU time
     probe, _ = time_oracle(cfg, sw, 1, 2)
-    seqs = max(1, min(cfg.B, int(120.0 / (min(probe) * (args.warmup + args.steps)))))
+    seqs = max(1, min(cfg.B, int(120.0 / (min(d + v for d, v in probe) * (args.warmup + args.steps)))))
     times, cores = time_oracle(cfg, sw, seqs, args.warmup + args.steps)
     timed = times[args.warmup:]
-    sec = sum(timed) / len(timed)
+    sec = sum(d + v for d, v in timed) / len(timed)
+    sec_d = sum(d for d, _ in timed) / len(timed)
+    sec_v = sum(v for _, v in timed) / len(timed)
     val = seqs / sec
     sample = f"{seqs} of {cfg.B} sequences of {cfg.name} per step (full tree + verify), plain C oracle, OpenMP"
     out = {
         "impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": sec * 1e3, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-        "config": {"workload": cfg.name, "B": cfg.B, "K": cfg.K, "n_heads": cfg.n, "topk": list(cfg.topk),
-                   "V": cfg.V, "d_base": cfg.d_base, "d_inner": cfg.d_inner},
-        "cpu_baseline": {"value": val, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+        "config": workload_config(cfg, max(1, args.gpus), logits_rotation(cfg)),
+        "cpu_baseline": {"value": val, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample,
+                         "draft": seqs / sec_d, "verify": seqs / sec_v},
         "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
     }
     print(json.dumps(out), flush=True)
+
+
+class Workload:
+    """One configuration resident in HBM: weights, a handle, draft inputs, rotating logits buffers, workspaces."""
+
+    def __init__(self, cfg, dev, B, synth, torch):
+        self.cfg, self.dev, self.B, self.torch = cfg, dev, B, torch
+        self.sw = synth.make_weights(cfg, device=dev)
+        self.h = B.spec_create(self.sw)
+        self.ctx, self.tok = synth.make_draft_inputs(cfg, device=dev)
+        n, K, Bn, V = cfg.n, cfg.K, cfg.B, cfg.V
+        self.ws = torch.empty(B.spec_draft_workspace_bytes(self.h, Bn, cfg.topk, K), dtype=torch.uint8, device=dev)
+        self.cand = torch.empty((Bn, K, n), dtype=torch.int32, device=dev)
+        self.logp = torch.empty((Bn, K), dtype=torch.float32, device=dev)
+        B.spec_draft(self.h, self.ctx, self.tok, cfg.topk, K, cand_tok=self.cand, cand_logp=self.logp, workspace=self.ws)
+        assert B.spec_poll_error(self.ws) == 0
+        # base-model logits: rotate over several distinct buffers so verify never re-reads a buffer that could
+        # still sit in the 126 MB L2; matches are planted at the tokens the draft proposes
+        self.logits_bytes = Bn * K * (n + 1) * V * 2
+        self.n_rot = logits_rotation(cfg)
+        self.rot = [synth.make_base_logits(dataclasses.replace(cfg, seed=cfg.seed + 100 * i), self.cand, device=dev)
+                    for i in range(self.n_rot)]
+        self.vws = torch.empty(B.spec_verify_workspace_bytes(Bn, K, n, V, B.SPEC_BF16), dtype=torch.uint8, device=dev)
+        self.acc = torch.empty(Bn, dtype=torch.int32, device=dev)
+        self.best = torch.empty(Bn, dtype=torch.int32, device=dev)
+        self.nxt = torch.empty(Bn, dtype=torch.int32, device=dev)
+
+    def draft(self, i=0):
+        c = self.cfg
+        self.B.spec_draft(self.h, self.ctx, self.tok, c.topk, c.K, cand_tok=self.cand, cand_logp=self.logp, workspace=self.ws)
+
+    def verify(self, i=0, early=False):
+        self.B.spec_verify(self.cand, self.rot[i % self.n_rot], accept_len=self.acc, best_cand=self.best,
+                           next_tok=self.nxt, workspace=self.vws, early_exit=early)
+
+    def step(self, i=0):
+        self.draft(i)
+        self.verify(i)
+
+    def close(self):
+        self.B.spec_destroy(self.h)
+        self.rot = self.sw = self.ws = None
+        self.torch.cuda.empty_cache()
+
+
+def time_loop(torch, fn, iters: int, warm: int = 3) -> float:
+    """Milliseconds per call of fn(i), CUDA events on the current stream, after `warm` untimed calls."""
+    stream = torch.cuda.current_stream()
+    for i in range(warm):
+        fn(i)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for i in range(iters):
+        fn(i)
+    e1.record(stream)
+    torch.cuda.synchronize()
+    return e0.elapsed_time(e1) / iters
+
+
+def head_alone(W: "Workload", level: int, rows: int, iters: int):
+    """The head GEMM of `level` with its fused epilogue alone (spec_head_partials), `rows` rows, launched back
+    to back: its weights (hundreds of MB) exceed L2, so nothing is re-read from there."""
+    torch, B, cfg = W.torch, W.B, W.cfg
+    k = cfg.topk[level]
+    g = torch.Generator(device=W.dev).manual_seed(5 + level)
+    S = (torch.randn(rows, cfg.d_inner, generator=g, device=W.dev) * 0.5).to(torch.bfloat16)
+    ws = torch.empty(B.spec_head_workspace_bytes(W.h, rows, k), dtype=torch.uint8, device=W.dev)
+    return time_loop(torch, lambda i: B.spec_head_partials(W.h, level, S, k, ws), iters)
+
+
+def head_roofline(cfg, rows: int, ms: float, peaks, traffic=None):
+    """Roofline entry of one head launch: below the ridge the weight stream bounds it, above it the tensor cores."""
+    flops = 2.0 * rows * cfg.d_inner * cfg.V
+    w_bytes = 2.0 * cfg.V * cfg.d_inner + 2.0 * rows * cfg.d_inner
+    ridge = peaks["bf16_tflops"] * 1e12 / (peaks["hbm_gbs"] * 1e9)
+    name = f"gemm_tc_kernel (vocabulary head: {rows} x {cfg.d_inner} x {cfg.V})"
+    if rows >= ridge:
+        ach = flops / (ms * 1e-3) / 1e12
+        return {"kernel": name, "bound": "tensor", "achieved": ach, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
+                "frac": ach / peaks["bf16_tflops"], "traffic": traffic, "peak_source": peaks["source"] + " burst",
+                "frac_of_sustained": ach / peaks["bf16_tflops_sustained"], "us": round(ms * 1e3, 2)}
+    ach = w_bytes / (ms * 1e-3) / 1e9
+    return {"kernel": name, "bound": "hbm", "achieved": ach, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+            "frac": ach / peaks["hbm_gbs"], "traffic": traffic, "peak_source": peaks["source"], "us": round(ms * 1e3, 2)}
+
+
+def verify_roofline(W: "Workload", ms: float, ms_early: float, peaks, traffic=None):
+    gbs = W.logits_bytes / (ms * 1e-3) / 1e9
+    return {"kernel": "verify_stream_kernel + verify_accept_kernel", "bound": "hbm", "achieved": gbs,
+            "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": gbs / peaks["hbm_gbs"], "peak_source": peaks["source"] + " copy bandwidth",
+            "frac_of_nameplate_8TBs": gbs / 8000.0, "traffic": traffic, "us": round(ms * 1e3, 2), "bytes": W.logits_bytes,
+            "early_exit_form_us": round(ms_early * 1e3, 2)}
+
+
+def workload_entry(W: "Workload", peaks, iters: int, world: int, shard):
+    """Step, draft and verify times of one workload and the roofline fractions of its dominant head and of verify."""
+    torch, cfg = W.torch, W.cfg
+    step_ms = time_loop(torch, W.step, iters)
+    draft_ms = time_loop(torch, W.draft, iters)
+    verify_ms = time_loop(torch, W.verify, iters)
+    early_ms = time_loop(torch, lambda i: W.verify(i, early=True), iters)
+    assert W.B.spec_poll_error(W.ws) == 0
+    last = cfg.n - 1
+    heads = []
+    for l in range(cfg.n):
+        ms = head_alone(W, l, cfg.nodes(l), max(5, iters // 2))
+        heads.append(head_roofline(cfg, cfg.nodes(l), ms, peaks))
+    tau = float(W.acc.float().mean().item()) + 1.0
+    return {"B": cfg.B, "K": cfg.K, "topk": list(cfg.topk), "V": cfg.V, "d_inner": cfg.d_inner, "steps_timed": iters,
+            "step_us": round(step_ms * 1e3, 2), "draft_us": round(draft_ms * 1e3, 2), "verify_us": round(verify_ms * 1e3, 2),
+            "verify_early_exit_us": round(early_ms * 1e3, 2),
+            "sequences_per_s": shard.whole_job_rate(cfg.B, world, step_ms * 1e-3),
+            "dominant_head": heads[last], "heads": [{"rows": cfg.nodes(l), "bound": hd["bound"], "us": hd["us"],
+                                                    "frac": round(hd["frac"], 3)} for l, hd in enumerate(heads)],
+            "verify_GBs": round(W.logits_bytes / (verify_ms * 1e-3) / 1e9, 1),
+            "verify_frac_of_measured_copy": round(W.logits_bytes / (verify_ms * 1e-3) / 1e9 / peaks["hbm_gbs"], 3),
+            "synthetic_tokens_per_step": tau}
 
 
 def run_only(args, cfg, peaks, dev):
@@ -226,6 +362,7 @@ def main():
     ap.add_argument("--config", default="llama2-13b")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--headline-only", action="store_true", help="skip the `workloads` entries of the other four shapes")
     ap.add_argument("--swap-max-rows", type=int, default=None,
                     help="--only head*: levels of at most this many rows use the weight-stream form (0: never)")
     ap.add_argument("--producers", type=int, default=0, help="--only head*: TMA-issuing threads per CTA (1 or 2)")
@@ -270,30 +407,13 @@ def main():
         return
 
     # ---------------------------------------------------------------- inputs, resident in HBM
-    sw = synth.make_weights(cfg, device=dev)
-    h = B.spec_create(sw)
-    ctx, tok = synth.make_draft_inputs(cfg, device=dev)
-    n, K, Bn, V = cfg.n, cfg.K, cfg.B, cfg.V
-    ws = torch.empty(B.spec_draft_workspace_bytes(h, Bn, cfg.topk, K), dtype=torch.uint8, device=dev)
-    cand = torch.empty((Bn, K, n), dtype=torch.int32, device=dev)
-    logp = torch.empty((Bn, K), dtype=torch.float32, device=dev)
-    B.spec_draft(h, ctx, tok, cfg.topk, K, cand_tok=cand, cand_logp=logp, workspace=ws)
-    assert B.spec_poll_error(ws) == 0
-    # base-model logits: rotate over several distinct buffers so verify never re-reads a buffer that
-    # could still sit in the 126 MB L2; matches are planted at the tokens the draft proposes
-    logits_bytes = Bn * K * (n + 1) * V * 2
-    n_rot = max(2, min(8, (512 << 20) // logits_bytes + 1))
-    rot = [synth.make_base_logits(dataclasses.replace(cfg, seed=cfg.seed + 100 * i), cand, device=dev)
-           for i in range(n_rot)]
-    vws = torch.empty(B.spec_verify_workspace_bytes(Bn, K, n, V, B.SPEC_BF16), dtype=torch.uint8, device=dev)
-    acc = torch.empty(Bn, dtype=torch.int32, device=dev)
-    best = torch.empty(Bn, dtype=torch.int32, device=dev)
-    nxt = torch.empty(Bn, dtype=torch.int32, device=dev)
+    W = Workload(cfg, dev, B, synth, torch)
+    h, n, K, Bn, V = W.h, cfg.n, cfg.K, cfg.B, cfg.V
+    ctx, tok, ws, cand, logp, rot, n_rot, vws = W.ctx, W.tok, W.ws, W.cand, W.logp, W.rot, W.n_rot, W.vws
+    acc, best, nxt = W.acc, W.best, W.nxt
+    logits_bytes = W.logits_bytes
     stream = torch.cuda.current_stream()
-
-    def step(i):
-        B.spec_draft(h, ctx, tok, cfg.topk, K, cand_tok=cand, cand_logp=logp, workspace=ws)
-        B.spec_verify(cand, rot[i % n_rot], accept_len=acc, best_cand=best, next_tok=nxt, workspace=vws)
+    step = W.step
 
     def barrier():
         if dist is not None:
@@ -303,25 +423,49 @@ def main():
     def max_over_ranks(x: float) -> float:
         return shard.max_over_ranks(x, dist, dev)
 
+    def timed_region(steps: int):
+        """`steps` steps between two events, a barrier and a synchronize on both sides, clocks sampled meanwhile."""
+        barrier()
+        sampler = ClockSampler(local_rank)
+        if rank == 0:
+            sampler.start()
+            time.sleep(0.25)
+        barrier()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for i in range(steps):
+            step(i)
+        e1.record(stream)
+        barrier()
+        ms = max_over_ranks(e0.elapsed_time(e1) / steps)
+        return ms, (sampler.stop() if rank == 0 else None)
+
     # ---------------------------------------------------------------- device-resident timing
     for i in range(args.warmup):
         step(i)
-    barrier()
-    sampler = ClockSampler(local_rank)
-    if rank == 0:
-        sampler.start()
-        time.sleep(0.25)
-    barrier()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e0.record(stream)
-    for i in range(args.steps):
-        step(i)
-    e1.record(stream)
-    barrier()
-    ms_step = max_over_ranks(e0.elapsed_time(e1) / args.steps)
-    clocks = sampler.stop() if rank == 0 else None
+    ms_step, clocks = timed_region(args.steps)
     assert B.spec_poll_error(ws) == 0
     tau = float(acc.float().mean().item()) + 1.0
+    # Which clock regime was that?  A region of a few milliseconds runs at boost clocks and is over before
+    # nvidia-smi has sampled twice; half a second of steps reaches the power-capped clocks.  When the timed
+    # region was short a second, long one is measured too and both are reported.
+    sustained = None
+    region_s = ms_step * 1e-3 * args.steps
+    if region_s < 0.5:
+        long_steps = int(0.6 / (ms_step * 1e-3)) + 1
+        ms_long, clocks_long = timed_region(long_steps)
+        sustained = {"steps": long_steps, "ms_per_step": ms_long, "value": shard.whole_job_rate(Bn, world, ms_long * 1e-3),
+                     "clocks": clocks_long}
+    regime = None
+    if rank == 0:
+        ck = clocks if sustained is None else sustained["clocks"]
+        regime = {"timed_region_s": round(region_s, 4),
+                  "kind": "sustained (half a second or more of back-to-back steps)" if region_s >= 0.5
+                          else "burst (a timed region of a few milliseconds: boost clocks; see `sustained`)",
+                  "sm_mhz_median": clocks["sm_mhz"], "clock_samples": clocks.get("samples"),
+                  "sw_power_cap_seen": "sw_power_cap" in (clocks.get("reasons") or []),
+                  "sustained_sm_mhz_median": ck["sm_mhz"], "sustained_clock_samples": ck.get("samples"),
+                  "sustained_sw_power_cap_seen": "sw_power_cap" in (ck.get("reasons") or [])}
 
     # ---------------------------------------------------------------- end to end from host buffers
     pin = lambda t: t.cpu().pin_memory()
@@ -354,6 +498,7 @@ def main():
         e2e_step(i)
     torch.cuda.synchronize()
     e2e_ms = max_over_ranks((time.perf_counter() - t0) * 1e3 / e2e_steps)
+    del d_logits, h_rot
 
     # ---------------------------------------------------------------- the same steps as one CUDA graph
     # n_rot steps (one per logits buffer) captured once and replayed: what is left when the host's launch
@@ -385,9 +530,22 @@ def main():
         sys.stderr.write(f"graph replay skipped: {e}\n")
     assert B.spec_poll_error(ws) == 0
 
+    # ---------------------------------------------------------------- host time of one spec_draft call
+    # CPU clock around the call alone (nothing is waited for): argument checks, the plan, the launches
+    torch.cuda.synchronize()
+    host_us = []
+    for i in range(30):
+        t0 = time.perf_counter()
+        W.draft(i)
+        host_us.append((time.perf_counter() - t0) * 1e6)
+        if i % 5 == 4:
+            torch.cuda.synchronize()
+    host_draft_us = statistics.median(host_us)
+    torch.cuda.synchronize()
+
     # ---------------------------------------------------------------- per-kernel times (CUDA events)
-    B.spec_set_option(h, B.SPEC_OPT_PROFILE, 1)
     prof_steps = max(3, min(args.steps, 50))
+    B.spec_set_option(h, B.SPEC_OPT_PROFILE, 1)
     sums = None
     for i in range(prof_steps):
         step(i)
@@ -395,59 +553,20 @@ def main():
         sums = ms if sums is None else [a + b for a, b in zip(sums, ms)]
     kern_ms = [s / prof_steps for s in sums]
     B.spec_set_option(h, B.SPEC_OPT_PROFILE, 0)
-    # verify alone, rotating buffers
-    v0, v1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    for i in range(3):
-        B.spec_verify(cand, rot[i % n_rot], accept_len=acc, best_cand=best, next_tok=nxt, workspace=vws)
-    torch.cuda.synchronize()
-    v0.record(stream)
-    for i in range(prof_steps):
-        B.spec_verify(cand, rot[i % n_rot], accept_len=acc, best_cand=best, next_tok=nxt, workspace=vws)
-    v1.record(stream)
-    torch.cuda.synchronize()
-    verify_ms = v0.elapsed_time(v1) / prof_steps
-    # the early-exit form on the same inputs (reads only the rows up to each candidate's first mismatch)
-    for i in range(3):
-        B.spec_verify(cand, rot[i % n_rot], accept_len=acc, best_cand=best, next_tok=nxt, workspace=vws, early_exit=True)
-    torch.cuda.synchronize()
-    v0.record(stream)
-    for i in range(prof_steps):
-        B.spec_verify(cand, rot[i % n_rot], accept_len=acc, best_cand=best, next_tok=nxt, workspace=vws, early_exit=True)
-    v1.record(stream)
-    torch.cuda.synchronize()
-    verify_early_ms = v0.elapsed_time(v1) / prof_steps
+    draft_ms = time_loop(torch, W.draft, prof_steps)
+    verify_ms = time_loop(torch, W.verify, prof_steps)
+    verify_early_ms = time_loop(torch, lambda i: W.verify(i, early=True), prof_steps)
 
-    # the vocabulary head alone at M = B*K rows (GEMM + merge kernels back to back), last head's weights
+    # every level's head alone at its own row count, and the last head at M = B*K rows (GEMM + merge kernels)
+    heads = [head_roofline(cfg, cfg.nodes(l), head_alone(W, l, cfg.nodes(l), prof_steps), peaks) for l in range(n)]
     bk_rows = Bn * K
     Sbk = (torch.randn(bk_rows, cfg.d_inner, generator=torch.Generator(device=dev).manual_seed(5), device=dev) * 0.5).to(torch.bfloat16)
     hk = cfg.topk[-1]
     htok = torch.empty((bk_rows, hk), dtype=torch.int32, device=dev)
     hlogp = torch.empty((bk_rows, hk), dtype=torch.float32, device=dev)
     hws = torch.empty(B.spec_head_workspace_bytes(h, bk_rows, hk), dtype=torch.uint8, device=dev)
-    for i in range(3):
-        B.spec_head_topk(h, n - 1, Sbk, hk, tok=htok, logp=hlogp, workspace=hws)
-    torch.cuda.synchronize()
-    v0.record(stream)
-    for i in range(prof_steps):
-        B.spec_head_topk(h, n - 1, Sbk, hk, tok=htok, logp=hlogp, workspace=hws)
-    v1.record(stream)
-    torch.cuda.synchronize()
-    bk_ms = v0.elapsed_time(v1) / prof_steps
-    # the dominant kernel alone: head GEMM of the last level with its fused epilogue, at that level's row
-    # count, launched back to back on the timed stream (262 MB of weights per launch: nothing stays in L2)
-    rows_dom = cfg.nodes(n - 1)
-    Sdom = Sbk[:rows_dom].contiguous() if rows_dom <= bk_rows else (
-        torch.randn(rows_dom, cfg.d_inner, generator=torch.Generator(device=dev).manual_seed(6), device=dev) * 0.5).to(torch.bfloat16)
-    dws = torch.empty(B.spec_head_workspace_bytes(h, rows_dom, hk), dtype=torch.uint8, device=dev)
-    for i in range(3):
-        B.spec_head_partials(h, n - 1, Sdom, hk, dws)
-    torch.cuda.synchronize()
-    v0.record(stream)
-    for i in range(prof_steps):
-        B.spec_head_partials(h, n - 1, Sdom, hk, dws)
-    v1.record(stream)
-    torch.cuda.synchronize()
-    head_alone_ms = v0.elapsed_time(v1) / prof_steps
+    bk_ms = time_loop(torch, lambda i: B.spec_head_topk(h, n - 1, Sbk, hk, tok=htok, logp=hlogp, workspace=hws), prof_steps)
+    del Sbk, hws
 
     # the same step with e4m3 copies of the heads attached (used by the levels of up to 128 nodes)
     B.spec_attach_fp8_heads(h)
@@ -455,19 +574,29 @@ def main():
 
     def step8(i):
         B.spec_draft(h, ctx, tok, cfg.topk, K, cand_tok=cand, cand_logp=logp, workspace=ws8)
-        B.spec_verify(cand, rot[i % n_rot], accept_len=acc, best_cand=best, next_tok=nxt, workspace=vws)
+        W.verify(i)
 
-    for i in range(3):
-        step8(i)
-    torch.cuda.synchronize()
-    v0.record(stream)
-    for i in range(prof_steps):
-        step8(i)
-    v1.record(stream)
-    torch.cuda.synchronize()
-    fp8_step_ms = v0.elapsed_time(v1) / prof_steps
+    fp8_step_ms = time_loop(torch, step8, prof_steps)
     assert B.spec_poll_error(ws8) == 0
     B.spec_detach_fp8_heads(h)
+    del ws8
+
+    # single-candidate drafts (K = 1, branching 1 everywhere: Sec. 4.2 / Sec. 5) at this workload's widths
+    k1 = {}
+    one = (1,) * n
+    for bk in (1, 16, 64):
+        c1 = dataclasses.replace(cfg, topk=one, K=1, B=bk)
+        ctx1, tok1 = synth.make_draft_inputs(c1, device=dev)
+        ws1 = torch.empty(B.spec_draft_workspace_bytes(h, bk, one, 1), dtype=torch.uint8, device=dev)
+        c_out = torch.empty((bk, 1, n), dtype=torch.int32, device=dev)
+        l_out = torch.empty((bk, 1), dtype=torch.float32, device=dev)
+        ms1 = time_loop(torch, lambda i: B.spec_draft(h, ctx1, tok1, one, 1, cand_tok=c_out, cand_logp=l_out, workspace=ws1),
+                        prof_steps)
+        assert B.spec_poll_error(ws1) == 0
+        w_bytes = sum(2.0 * V * cfg.d_inner + 2.0 * cfg.d_inner * cfg.d_in(l) for l in range(n))
+        k1[f"B={bk}"] = {"draft_us": round(ms1 * 1e3, 2), "launches": 2 + 2 * n,
+                         "weight_stream_floor_us": round(w_bytes / (peaks["hbm_gbs"] * 1e9) * 1e6, 1),
+                         "frac_of_hbm_floor": round(w_bytes / (peaks["hbm_gbs"] * 1e9) / (ms1 * 1e-3), 3)}
 
     if rank != 0:
         if dist is not None:
@@ -479,67 +608,76 @@ def main():
         names += [f"proj_gemm[{l}]", f"mix_ln_gelu[{l}]", f"head_gemm[{l}]", f"merge_expand[{l}]"]
     names.append("prune")
     kernels = {nm: round(ms * 1e3, 2) for nm, ms in zip(names, kern_ms)}      # microseconds
-    # dominant kernel: the vocabulary-head GEMM of the last (widest) level
+    # dominant kernel: the vocabulary-head GEMM of the last (widest) level, alone, back to back
     rows_last = cfg.nodes(n - 1)
-    head_ms = head_alone_ms   # average launch duration of the kernel itself (the per-kernel list below brackets
-                              # every launch with events, which adds 2-3 us)
-    flops = 2.0 * rows_last * cfg.d_inner * V
-    w_bytes = 2.0 * V * cfg.d_inner + 2.0 * rows_last * cfg.d_inner
-    ridge = peaks["bf16_tflops"] * 1e12 / (peaks["hbm_gbs"] * 1e9)
-    if rows_last >= ridge:
-        ach = flops / (head_ms * 1e-3) / 1e12
-        roof = {"kernel": f"gemm_tc_kernel (vocabulary head, level {n - 1}: {rows_last} x {cfg.d_inner} x {V})",
-                "bound": "tensor", "achieved": ach, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
-                "frac": ach / peaks["bf16_tflops"], "traffic": NCU_TRAFFIC_BYTES.get((cfg.name, f"head_gemm_{rows_last}_rows")),
-                "peak_source": peaks["source"] + " burst",
-                "frac_of_sustained": ach / peaks["bf16_tflops_sustained"]}
-    else:
-        ach = w_bytes / (head_ms * 1e-3) / 1e9
-        roof = {"kernel": f"gemm_tc_kernel (vocabulary head, level {n - 1}: {rows_last} x {cfg.d_inner} x {V})",
-                "bound": "hbm", "achieved": ach, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                "frac": ach / peaks["hbm_gbs"], "traffic": None, "peak_source": peaks["source"]}
-    v_gbs = logits_bytes / (verify_ms * 1e-3) / 1e9
-    roof_verify = {"kernel": "verify_stream_kernel + verify_accept_kernel", "bound": "hbm", "achieved": v_gbs,
-                   "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": v_gbs / peaks["hbm_gbs"],
-                   "traffic": NCU_TRAFFIC_BYTES.get((cfg.name, "verify_stream")),
-                   "us": round(verify_ms * 1e3, 2), "bytes": logits_bytes,
-                   "early_exit_form_us": round(verify_early_ms * 1e3, 2)}
-    # heads below the ridge are weight-bandwidth bound: report their HBM fraction too
-    head_hbm = {}
-    for l in range(n):
-        hb = 2.0 * V * cfg.d_inner + 2.0 * cfg.nodes(l) * cfg.d_inner
-        head_hbm[f"head_gemm[{l}]"] = {"rows": cfg.nodes(l),
-                                       "GB/s": round(hb / (kern_ms[4 * l + 2] * 1e-3) / 1e9, 1),
-                                       "TFLOP/s": round(2.0 * cfg.nodes(l) * cfg.d_inner * V / (kern_ms[4 * l + 2] * 1e-3) / 1e12, 1)}
+    roof = dict(heads[n - 1])
+    roof["traffic"] = NCU_TRAFFIC_BYTES.get((cfg.name, f"head_gemm_{rows_last}_rows"))
+    roof_verify = verify_roofline(W, verify_ms, verify_early_ms, peaks, NCU_TRAFFIC_BYTES.get((cfg.name, "verify_stream")))
+    head_list = {f"head_gemm[{l}]": {"rows": cfg.nodes(l), "bound": hd["bound"], "us": hd["us"], "unit": hd["unit"],
+                                     "achieved": round(hd["achieved"], 1), "frac": round(hd["frac"], 3)}
+                 for l, hd in enumerate(heads)}
 
+    # ---------------------------------------------------------------- the other workloads (1 GPU only)
+    workloads = {cfg.name: {"B": Bn, "K": K, "topk": list(cfg.topk), "V": V, "d_inner": cfg.d_inner, "steps_timed": args.steps,
+                            "step_us": round(ms_step * 1e3, 2), "draft_us": round(draft_ms * 1e3, 2),
+                            "verify_us": round(verify_ms * 1e3, 2), "verify_early_exit_us": round(verify_early_ms * 1e3, 2),
+                            "sequences_per_s": shard.whole_job_rate(Bn, world, ms_step * 1e-3), "dominant_head": roof,
+                            "heads": [{"rows": cfg.nodes(l), "bound": hd["bound"], "us": hd["us"], "frac": round(hd["frac"], 3)}
+                                      for l, hd in enumerate(heads)],
+                            "verify_GBs": round(roof_verify["achieved"], 1),
+                            "verify_frac_of_measured_copy": round(roof_verify["frac"], 3),
+                            "synthetic_tokens_per_step": tau, "host_us_per_spec_draft_call": round(host_draft_us, 1)}}
     cpu = None
-    if world == 1 and not args.no_cpu_baseline:
-        sw_cpu = synth.SpecWeights(cfg, *[[t.cpu() for t in lst] for lst in (sw.emb, sw.proj, sw.ln_gamma, sw.ln_beta, sw.head)],
-                                   sw.state_weight, sw.emb_weight, sw.ln_eps)
-        # about 15 s of oracle time: one sequence first to size the sample, then whole passes over as
-        # many sequences of the batch as fit
-        probe, cores = time_oracle(cfg, sw_cpu, 1, 2)
-        seqs = max(1, min(Bn, int(15.0 / min(probe))))
-        one_pass, cores = time_oracle(cfg, sw_cpu, seqs, 1)
-        reps = max(1, min(12, int(round(15.0 / one_pass[0])) - 1))
-        times, cores = time_oracle(cfg, sw_cpu, seqs, reps)
-        times = one_pass + times
-        cpu = {"value": seqs * len(times) / sum(times), "unit": UNIT, "cores": cores, "kind": "oracle",
-               "sample": f"{seqs} of {Bn} sequences of {cfg.name} (full draft tree + verify) x {len(times)} passes, "
-                         f"{sum(times):.1f} s of oracle time"}
+    if world == 1:
+        sw_cpu = None
+        if not args.no_cpu_baseline:
+            sw_cpu = synth.SpecWeights(cfg, *[[t.cpu() for t in lst] for lst in (W.sw.emb, W.sw.proj, W.sw.ln_gamma, W.sw.ln_beta, W.sw.head)],
+                                       W.sw.state_weight, W.sw.emb_weight, W.sw.ln_eps)
+        W.close()
+        if not args.headline_only:
+            for name, c in synth.CONFIGS.items():
+                if name == cfg.name:
+                    continue
+                Wo = Workload(c, dev, B, synth, torch)
+                est = time_loop(torch, Wo.step, 3)
+                iters = max(5, min(args.steps, 200, int(150.0 / est) + 1))     # about 0.15 s per timed loop
+                entry = workload_entry(Wo, peaks, iters, world, shard)
+                torch.cuda.synchronize()
+                hu = []
+                for i in range(10):
+                    t0 = time.perf_counter()
+                    Wo.draft(i)
+                    hu.append((time.perf_counter() - t0) * 1e6)
+                torch.cuda.synchronize()
+                entry["host_us_per_spec_draft_call"] = round(statistics.median(hu), 1)
+                workloads[name] = entry
+                Wo.close()
+                del Wo
+        if sw_cpu is not None:
+            # about 15 s of oracle time: one sequence first to size the sample, then whole passes over as
+            # many sequences of the batch as fit
+            probe, cores = time_oracle(cfg, sw_cpu, 1, 2)
+            seqs = max(1, min(Bn, int(15.0 / min(d + v for d, v in probe))))
+            one_pass, cores = time_oracle(cfg, sw_cpu, seqs, 1)
+            reps = max(1, min(12, int(round(15.0 / sum(one_pass[0]))) - 1))
+            times, cores = time_oracle(cfg, sw_cpu, seqs, reps)
+            times = one_pass + times
+            t_d, t_v = sum(d for d, _ in times), sum(v for _, v in times)
+            cpu = {"value": seqs * len(times) / (t_d + t_v), "unit": UNIT, "cores": cores, "kind": "oracle",
+                   "draft": seqs * len(times) / t_d, "verify": seqs * len(times) / t_v,
+                   "sample": f"{seqs} of {Bn} sequences of {cfg.name} (full draft tree + verify) x {len(times)} passes, "
+                             f"{t_d + t_v:.1f} s of oracle time; `draft` and `verify` are the two parts timed apart, `value` both"}
 
-    # per step: header init, level-0 projection, then per level mix, head GEMM (the next level's projection
-    # rides in the same launch) and merge (the last one also prunes); verify = streaming arg-max + accept
-    launches_per_step = 1 + 1 + 3 * n + 2
+    # per step: level-0 projection (clears the header), then per level mix, head GEMM (the next level's
+    # projection rides in the same launch) and merge (the last one also prunes); verify = streaming arg-max + accept
+    launches_per_step = 1 + 3 * n + 2
     out = {
         "metric": METRIC, "value": shard.whole_job_rate(Bn, world, ms_step * 1e-3), "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-        "config": {"workload": cfg.name, "B": Bn, "K": K, "n_heads": n, "topk": list(cfg.topk), "V": V,
-                   "d_base": cfg.d_base, "d_inner": cfg.d_inner, "logits_dtype": "bf16",
-                   "l2": f"weights 1.7 GB+ per step exceed L2; verify rotates over {n_rot} distinct logits buffers",
-                   "parallelism": f"replicas x{world}, sequences independent, no collective"},
-        "roofline": roof, "roofline_verify": roof_verify, "head_gemms": head_hbm,
+        "config": workload_config(cfg, world, n_rot),
+        "roofline": roof, "roofline_verify": roof_verify, "head_gemms": head_list,
+        "head_gemms_note": "each level's head GEMM with its fused epilogue alone (spec_head_partials), back to back",
         "head_at_BK_rows": {"rows": bk_rows, "us": round(bk_ms * 1e3, 2), "what": "spec_head_topk: head GEMM + merge",
                             "TFLOP/s": round(2.0 * bk_rows * cfg.d_inner * V / (bk_ms * 1e-3) / 1e12, 1),
                             "frac_of_burst": round(2.0 * bk_rows * cfg.d_inner * V / (bk_ms * 1e-3) / 1e12 / peaks["bf16_tflops"], 3)},
@@ -547,8 +685,11 @@ def main():
                                  "what": "optional mode: e4m3 head copies on the weight-bound levels, short list re-scored in bf16"},
         "graph_replay": {"ms_per_step": None if graph_ms is None else round(graph_ms, 5),
                          "what": "the same draft + verify steps captured in one CUDA graph and replayed"},
-        "kernel_us": kernels, "kernel_us_note": "separate-kernel form bracketed by events (adds 2-3 us per kernel); "
-                                                "the timed step launches the next level's projection with the head",
+        "kernel_us": kernels, "kernel_us_note": "separate-kernel form bracketed by events (adds 2-3 us per kernel and takes "
+                                                "away the overlap of consecutive kernels); the timed step launches the next "
+                                                "level's projection with the head",
+        "k1": k1, "k1_note": f"spec_draft with K = 1 and branching 1 at every head, widths of {cfg.name}",
+        "workloads": workloads, "regime": regime, "sustained": sustained,
         "cpu_baseline": cpu,
         "e2e": {"value": shard.whole_job_rate(Bn, world, e2e_ms * 1e-3), "unit": UNIT, "ms_per_step": e2e_ms,
                 "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
