@@ -205,14 +205,18 @@ __device__ __forceinline__ void mix_ln_gelu_row(const MixArgs &m, int r, int tid
 }
 
 // (value desc, token id asc) ordering of candidates.
-__device__ __forceinline__ bool better(float v, int i, float w, int j) { return v > w || (v == w && i < j); }
+// Written without short-circuit operators and the exchanges below as selects: with "||" / "&&" and an "if"
+// around the swap every comparison became a data-dependent branch that diverges inside the warp, and one
+// 8-entry list took 2000-6000 cycles to fold instead of a few hundred.
+__device__ __forceinline__ bool better(float v, int i, float w, int j) { return (v > w) | ((v == w) & (i < j)); }
 
 // The pair at (va, ia) and the pair at (vb, ib) swap places unless the first is already the better one.
 __device__ __forceinline__ void order_pair(float &va, int &ia, float &vb, int &ib) {
-    if (better(vb, ib, va, ia)) {
-        const float fv = va; va = vb; vb = fv;
-        const int fi = ia; ia = ib; ib = fi;
-    }
+    const bool sw = better(vb, ib, va, ia);
+    const float hv = sw ? vb : va, lv = sw ? va : vb;
+    const int hi = sw ? ib : ia, li = sw ? ia : ib;
+    va = hv; vb = lv;
+    ia = hi; ib = li;
 }
 
 // Order-preserving map of a float (no NaN) onto unsigned integers, and back.
@@ -236,10 +240,9 @@ __device__ __forceinline__ void fold_tile_list(float (&tv)[SPEC_MAX_TOPK], int (
     int li[kT] = {i0.x, i0.y, i0.z, i0.w, i1.x, i1.y, i1.z, i1.w};
 #pragma unroll
     for (int j = 0; j < kT; ++j) {
-        if (j >= topk || !valid) {   // slots past the list's length hold nothing
-            lv[j] = -INFINITY;
-            li[j] = 0x7fffffff;
-        }
+        const bool none = (j >= topk) | !valid;   // slots past the list's length hold nothing
+        lv[j] = none ? -INFINITY : lv[j];
+        li[j] = none ? 0x7fffffff : li[j];
     }
     // 19-comparator sorting network for 8 inputs
 #define SPEC_CX(a, b) order_pair(lv[a], li[a], lv[b], li[b])
@@ -252,10 +255,9 @@ __device__ __forceinline__ void fold_tile_list(float (&tv)[SPEC_MAX_TOPK], int (
 #undef SPEC_CX
 #pragma unroll
     for (int j = 0; j < kT; ++j) {
-        if (better(lv[kT - 1 - j], li[kT - 1 - j], tv[j], ti[j])) {
-            tv[j] = lv[kT - 1 - j];
-            ti[j] = li[kT - 1 - j];
-        }
+        const bool take = better(lv[kT - 1 - j], li[kT - 1 - j], tv[j], ti[j]);
+        tv[j] = take ? lv[kT - 1 - j] : tv[j];
+        ti[j] = take ? li[kT - 1 - j] : ti[j];
     }
 #pragma unroll
     for (int stride = kT / 2; stride > 0; stride >>= 1) {
@@ -510,7 +512,7 @@ struct LeafKey {
 };
 
 __device__ __forceinline__ bool leaf_before(const LeafKey &a, const LeafKey &b) {
-    return a.score > b.score || (a.score == b.score && a.leaf < b.leaf);
+    return (a.score > b.score) | ((a.score == b.score) & (a.leaf < b.leaf));
 }
 
 // Writes candidate `rank` of sequence b: its score and the tokens on the path from the root to `leaf`.

@@ -605,7 +605,8 @@ struct SwapRun {
     int ti[SPEC_MAX_TOPK];
 };
 
-__device__ __forceinline__ bool cand_better(float v, int i, float w, int j) { return v > w || (v == w && i < j); }
+// (no short-circuit operators: every comparison would be a divergent branch)
+__device__ __forceinline__ bool cand_better(float v, int i, float w, int j) { return (v > w) | ((v == w) & (i < j)); }
 
 // Branch-free insertion into the sorted list: slot j takes its left neighbour when the newcomer beats that
 // neighbour, the newcomer when it beats only slot j, and keeps its entry otherwise.
@@ -712,18 +713,20 @@ __device__ __forceinline__ void merge_sorted8(SwapRun &r, const float (&ov)[SPEC
     static_assert(kT == 8, "three stages sort eight entries");
 #pragma unroll
     for (int j = 0; j < kT; ++j) {
-        if (cand_better(ov[kT - 1 - j], oi[kT - 1 - j], r.tv[j], r.ti[j])) {
-            r.tv[j] = ov[kT - 1 - j];
-            r.ti[j] = oi[kT - 1 - j];
-        }
+        const bool take = cand_better(ov[kT - 1 - j], oi[kT - 1 - j], r.tv[j], r.ti[j]);
+        r.tv[j] = take ? ov[kT - 1 - j] : r.tv[j];
+        r.ti[j] = take ? oi[kT - 1 - j] : r.ti[j];
     }
 #pragma unroll
     for (int stride = kT / 2; stride > 0; stride >>= 1) {
 #pragma unroll
         for (int j = 0; j < kT; ++j) {
-            if ((j & stride) == 0 && cand_better(r.tv[j + stride], r.ti[j + stride], r.tv[j], r.ti[j])) {
-                const float fv = r.tv[j]; r.tv[j] = r.tv[j + stride]; r.tv[j + stride] = fv;
-                const int fi = r.ti[j]; r.ti[j] = r.ti[j + stride]; r.ti[j + stride] = fi;
+            if ((j & stride) == 0) {   // (compile-time condition: the loops are unrolled)
+                const bool sw = cand_better(r.tv[j + stride], r.ti[j + stride], r.tv[j], r.ti[j]);
+                const float hv = sw ? r.tv[j + stride] : r.tv[j], lv = sw ? r.tv[j] : r.tv[j + stride];
+                const int hi = sw ? r.ti[j + stride] : r.ti[j], li = sw ? r.ti[j] : r.ti[j + stride];
+                r.tv[j] = hv; r.tv[j + stride] = lv;
+                r.ti[j] = hi; r.ti[j + stride] = li;
             }
         }
     }

@@ -75,10 +75,9 @@ __device__ __forceinline__ void warp_argmax(float &best, int &idx) {
     for (int off = 16; off > 0; off >>= 1) {
         float ob = __shfl_xor_sync(0xffffffffu, best, off);
         int oi = __shfl_xor_sync(0xffffffffu, idx, off);
-        if (ob > best || (ob == best && oi < idx)) {
-            best = ob;
-            idx = oi;
-        }
+        const bool take = (ob > best) | ((ob == best) & (oi < idx));
+        best = take ? ob : best;
+        idx = take ? oi : idx;
     }
 }
 
