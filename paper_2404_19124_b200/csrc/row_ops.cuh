@@ -528,13 +528,35 @@ __device__ __forceinline__ void emit_candidate(const PruneArgs &pa, int L, int K
     }
 }
 
+// Tokens on the path from the root to `leaf` of sequence b, requested together (their addresses depend on the
+// leaf index only, not on one another).
+__device__ __forceinline__ void load_path(const PruneArgs &pa, int L, int b, int leaf, int32_t (&path)[SPEC_MAX_HEADS]) {
+    int idx = leaf, per_seq = L;
+#pragma unroll
+    for (int l = SPEC_MAX_HEADS - 1; l >= 0; --l) {
+        if (l < pa.n) {
+            path[l] = __ldcg(pa.tok[l] + (size_t)b * per_seq + idx);
+            idx /= pa.topk[l];
+            per_seq /= pa.topk[l];
+        }
+    }
+}
+
 // Sequence b: the K best leaves by (score desc, leaf index asc), traced back to the root.  `keys`:
 // shared memory for Lpad entries, Lpad the power of two >= max(L, 2).  Up to 256 leaves every thread
-// counts how many leaves precede its own (that is its rank; no barriers); longer lists are sorted
-// bitonically.
+// counts how many leaves precede its own (that is its rank; no barriers) and has requested the tokens of its
+// own leaves' paths together with the scores, so a kept leaf is written out without another trip to memory;
+// longer lists are sorted bitonically.
 template <int kThreads, typename Sync>
 __device__ __forceinline__ void prune_sequence(const float *leaf_score, const PruneArgs &pa, int L, int Lpad, int K,
                                                int32_t *cand_tok, float *cand_logp, int b, int tid, LeafKey *keys) {
+    constexpr int kOwn = 256 / kThreads > 0 ? 256 / kThreads : 1;   // leaves per thread in the ranked form
+    int32_t path[kOwn][SPEC_MAX_HEADS];
+    if (L <= 256) {
+#pragma unroll
+        for (int q = 0; q < kOwn; ++q)
+            if (tid + q * kThreads < L) load_path(pa, L, b, tid + q * kThreads, path[q]);
+    }
     Sync::sync();   // a previous call may still be reading the keys
     for (int i = tid; i < Lpad; i += kThreads) {
         keys[i].score = (i < L) ? __ldcg(leaf_score + (size_t)b * L + i) : -INFINITY;
@@ -542,11 +564,19 @@ __device__ __forceinline__ void prune_sequence(const float *leaf_score, const Pr
     }
     Sync::sync();
     if (L <= 256) {
-        for (int i = tid; i < L; i += kThreads) {
+#pragma unroll
+        for (int q = 0; q < kOwn; ++q) {
+            const int i = tid + q * kThreads;
+            if (i >= L) continue;
             const LeafKey mine = keys[i];
             int rank = 0;
             for (int j = 0; j < L; ++j) rank += leaf_before(keys[j], mine) ? 1 : 0;
-            if (rank < K) emit_candidate(pa, L, K, cand_tok, cand_logp, b, rank, mine.score, mine.leaf);
+            if (rank < K) {
+                cand_logp[(size_t)b * K + rank] = mine.score;
+#pragma unroll
+                for (int l = 0; l < SPEC_MAX_HEADS; ++l)
+                    if (l < pa.n) cand_tok[((size_t)b * K + rank) * pa.n + l] = path[q][l];
+            }
         }
         return;
     }
@@ -577,15 +607,16 @@ template <int kThreads, typename Sync>
 __device__ __forceinline__ void prune_if_last(const MergeArgs &g, int r, int tid, LeafKey *keys, int *flag) {
     if (g.seq_done == nullptr) return;
     const int b = r / g.rows_per_seq;
-    __threadfence();
-    Sync::sync();
-    if (tid == 0) {
-        __threadfence();
-        *flag = (atomicAdd(g.seq_done + b, 1) == g.rows_per_seq - 1) ? 1 : 0;
+    if (g.rows_per_seq > 1) {   // (a sequence of one row is complete with this CTA's own children)
+        __threadfence();        // this CTA's children before its count
+        Sync::sync();
+        if (tid == 0) *flag = (atomicAdd(g.seq_done + b, 1) == g.rows_per_seq - 1) ? 1 : 0;
+        Sync::sync();
+        if (*flag == 0) return;
+        __threadfence();        // the other CTAs' children after the last count
+    } else {
+        Sync::sync();
     }
-    Sync::sync();
-    if (*flag == 0) return;
-    __threadfence();
     prune_sequence<kThreads, Sync>(g.score_out, g.prune, g.L, g.Lpad, g.K, g.cand_tok, g.cand_logp, b, tid, keys);
 }
 
