@@ -598,6 +598,30 @@ def main():
                          "weight_stream_floor_us": round(w_bytes / (peaks["hbm_gbs"] * 1e9) * 1e6, 1),
                          "frac_of_hbm_floor": round(w_bytes / (peaks["hbm_gbs"] * 1e9) / (ms1 * 1e-3), 3)}
 
+    # ---------------------------------------------------------------- vocabulary-parallel heads (N > 1 only)
+    # The optional mode for small batches: every rank holds 1/N of each head's vocabulary rows, the per-level
+    # lists are all-gathered with NCCL (no multicast loads anywhere), every rank ends with the same candidates.
+    # Whole-draft time with the exchange inside, max over ranks; never part of `value`.
+    vocab_parallel = None
+    if dist is not None:
+        try:
+            parts = shard.split_vocab(V, world)
+            lo, cnt = parts[rank]
+            wsh = dataclasses.replace(W.sw, head=[t[lo:lo + cnt].contiguous() for t in W.sw.head])
+            hv = B.spec_create(wsh, vocab_shard=(rank, world, lo))
+            wsv = torch.empty(B.spec_draft_workspace_bytes(hv, Bn, cfg.topk, K), dtype=torch.uint8, device=dev)
+            cv = torch.empty((Bn, K, n), dtype=torch.int32, device=dev)
+            lv = torch.empty((Bn, K), dtype=torch.float32, device=dev)
+            vp = lambda i: shard.draft_vocab_parallel(B, hv, ctx, tok, cfg.topk, K, workspace=wsv, cand_tok=cv, cand_logp=lv)
+            vp_ms = max_over_ranks(time_loop(torch, vp, max(3, min(args.steps, 50))))
+            same = bool(torch.equal(cv, cand))
+            vocab_parallel = {"draft_us": round(vp_ms * 1e3, 2), "ranks": world, "unsplit_draft_us": round(draft_ms * 1e3, 2),
+                              "same_candidates_as_unsplit_on_rank0": same,
+                              "what": "heads split by vocabulary rows over the ranks, NCCL all-gather of the per-level lists included"}
+            B.spec_destroy(hv)
+        except Exception as e:      # the optional mode must not take the scaling line down with it
+            vocab_parallel = {"error": repr(e)[:300]}
+
     if rank != 0:
         if dist is not None:
             dist.destroy_process_group()
@@ -689,7 +713,7 @@ def main():
                                                 "away the overlap of consecutive kernels); the timed step launches the next "
                                                 "level's projection with the head",
         "k1": k1, "k1_note": f"spec_draft with K = 1 and branching 1 at every head, widths of {cfg.name}",
-        "workloads": workloads, "regime": regime, "sustained": sustained,
+        "workloads": workloads, "regime": regime, "sustained": sustained, "vocab_parallel": vocab_parallel,
         "cpu_baseline": cpu,
         "e2e": {"value": shard.whole_job_rate(Bn, world, e2e_ms * 1e-3), "unit": UNIT, "ms_per_step": e2e_ms,
                 "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},

@@ -251,6 +251,13 @@ int spec_verify_static(const int32_t *cand_tok, const void *base_logits, int log
  *                            slot g lies at offset + g * slot_bytes.  A slot is fp32 [N_l, topk[l]] logits,
  *                            int32 [N_l, topk[l]] token ids, fp32 [N_l] log-sum-exp over the shard, padded
  *                            to 256 bytes.
+ *                            ORDER ACROSS RANKS: all levels use the same region at the same offset, with a slot
+ *                            size that changes from level to level.  A rank's region may therefore receive
+ *                            level l + 1 slots only after its own spec_draft_vp_merge(level l) has completed.
+ *                            A collective enqueued on the draft's stream (NCCL all-gather) orders this by
+ *                            itself; with direct peer stores the writer must first learn (an event, a flag, a
+ *                            barrier per level) that the peer's merge of the previous level is done.  Peer
+ *                            traffic is plain loads / stores or NCCL; the library issues no multicast loads.
  *   spec_draft_vp_local / _merge  arguments as spec_draft; the same B, topk, K and workspace for every
  *                            step of one draft (workspace size: spec_draft_workspace_bytes on the sharded
  *                            handle).  cand_tok / cand_logp are written by the merge of the last level

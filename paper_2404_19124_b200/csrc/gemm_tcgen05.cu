@@ -71,6 +71,7 @@ gemm_tc_kernel(const __grid_constant__ GemmMaps maps, const __grid_constant__ Ge
             AccPos ap{0, 0u};
             bool ok = true;
             for (int q = 0; ok && q < p.n_jobs; ++q) ok = mma_job(pp, p.job[q], rp, ap);
+            if (!ok || pp.bars->abort_flag) mma_drain(pp);
         }
     } else {
         AccPos ap{0, 0u};

@@ -50,6 +50,7 @@ struct __align__(8) Barriers {
     uint64_t empty[kMaxStages];
     uint64_t acc_full[2];
     uint64_t acc_empty[2];
+    uint64_t drained;           // abort path only: completes when every MMA issued so far has finished
     uint32_t tmem_base;
     volatile int abort_flag;
     volatile int epi_ok;        // mode 3: the epilogue leader's verdict on its wait, read by the other epilogue warps
@@ -224,6 +225,7 @@ __device__ __forceinline__ Pipe pipe_setup(uint8_t *smem_raw, int stages, uint32
             mbar_init(&pp.bars->acc_full[a], 1);
             mbar_init(&pp.bars->acc_empty[a], 4);   // one arrival per epilogue warp
         }
+        mbar_init(&pp.bars->drained, 1);
         pp.bars->abort_flag = 0;
         pp.bars->epi_ok = 1;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -459,6 +461,16 @@ __device__ __forceinline__ bool mma_job_kind(const Pipe &pp, const GemmJob &j, R
         if (++ap.acc == 2) { ap.acc = 0; ap.phase ^= 1u; }
     }
     return true;
+}
+
+// After a failed wait in any role: the MMAs issued so far may still be reading shared memory and writing
+// TMEM.  A commit tracks every tcgen05.mma this thread issued before it; its arrival on a barrier of its own
+// is waited for (bounded) before the CTA frees TMEM and gives up its shared memory.  Order at tear-down:
+// producers wait for their copies (producer_drain), this thread for its MMAs, then all threads meet at the
+// barrier in pipe_teardown and only then TMEM is deallocated.
+__device__ __forceinline__ void mma_drain(const Pipe &pp) {
+    umma_commit(&pp.bars->drained);
+    for (uint32_t it = 0; it < (1u << 20) && !mbar_try_wait(&pp.bars->drained, 0u); ++it) __nanosleep(32);
 }
 
 __device__ __forceinline__ bool mma_job(const Pipe &pp, const GemmJob &j, RingPos &rp, AccPos &ap) {

@@ -81,11 +81,21 @@ def split_vocab(V: int, world: int, multiple: int = 8) -> List[Tuple[int, int]]:
     return out
 
 
+_send_buffers = {}   # (device, bytes) -> uint8 tensor: the copy of this rank's slot that is sent, kept between calls
+
+
 def all_gather_slots(region, rank: int, dist, group=None) -> None:
     """`region`: uint8 tensor [world, slot_bytes] of which row `rank` is filled; afterwards every row is.
-    Any backend (NCCL on the GPU the region lives on, gloo for CPU tensors)."""
-    world = region.shape[0]
-    mine = region[rank].clone()
+    Any backend (NCCL on the GPU the region lives on, gloo for CPU tensors).  The slot that is sent is copied
+    into a buffer that is allocated once per (device, size) and reused, so a draft allocates nothing per level."""
+    import torch
+    world, nbytes = region.shape[0], region.shape[1]
+    key = (str(region.device), int(nbytes))
+    mine = _send_buffers.get(key)
+    if mine is None:
+        mine = torch.empty(nbytes, dtype=torch.uint8, device=region.device)
+        _send_buffers[key] = mine
+    mine.copy_(region[rank])
     dist.all_gather([region[g] for g in range(world)], mine, group=group)
 
 
