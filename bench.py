@@ -38,8 +38,8 @@ UNIT = "sequences/s"
 DEFAULT_STEPS, DEFAULT_WARMUP = 2000, 50
 
 NCU_TRAFFIC_BYTES = {
-    ("llama2-13b", "head_gemm_384_rows"): 278.9e6,     # profiles/gemm_tc_kernel_head_llama2-13b.md
-    ("llama2-13b", "verify_stream"): 135.2e6,          # profiles/verify_stream_kernel_llama2-13b.md
+    ("llama2-13b", "head_gemm_384_rows"): 279.2e6,     # profiles/gemm_tc_kernel_head_llama2-13b.md
+    ("llama2-13b", "verify_stream"): 134.9e6,          # profiles/verify_stream_kernel_llama2-13b.md
 }
 
 
