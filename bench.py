@@ -316,6 +316,8 @@ def run_only(args, cfg, peaks, dev):
             B.spec_set_option(h, B.SPEC_OPT_HEAD_SWAP_MAX_ROWS, args.swap_max_rows)
         if args.producers:
             B.spec_set_option(h, B.SPEC_OPT_GEMM_PRODUCERS, args.producers)
+        if args.pair is not None:
+            B.spec_set_option(h, B.SPEC_OPT_HEAD_PAIR, args.pair)
         g = torch.Generator(device=dev).manual_seed(5)
         S = (torch.randn(rows, cfg.d_inner, generator=g, device=dev) * 0.5).to(torch.bfloat16)
         tok = torch.empty((rows, k), dtype=torch.int32, device=dev)
@@ -365,6 +367,7 @@ def main():
     ap.add_argument("--headline-only", action="store_true", help="skip the `workloads` entries of the other four shapes")
     ap.add_argument("--swap-max-rows", type=int, default=None,
                     help="--only head*: levels of at most this many rows use the weight-stream form (0: never)")
+    ap.add_argument("--pair", type=int, default=None, help="--only head*: 1 = CTA pairs for more than 128 rows, 0 = one CTA per tile")
     ap.add_argument("--producers", type=int, default=0, help="--only head*: TMA-issuing threads per CTA (1 or 2)")
     ap.add_argument("--vocab", type=int, default=None, help="--only head*: vocabulary size instead of the workload's")
     ap.add_argument("--topk", type=int, default=None, help="--only head*: branching factor (default: the last level's)")

@@ -65,8 +65,13 @@ enum spec_option {
                                   -1 (default) = automatic: up to 8 nodes, or up to 32 when the
                                   vocabulary gives every CTA at least four 128-row tiles.  Ignored
                                   while SPEC_OPT_HEAD_BLOCK_N forces a tile width.              */
-    SPEC_OPT_GEMM_PRODUCERS = 6  /* 1 or 2 (default) threads per CTA issue the TMA copies of the GEMM
+    SPEC_OPT_GEMM_PRODUCERS = 6, /* 1 or 2 (default) threads per CTA issue the TMA copies of the GEMM
                                   kernels; process-wide, not per handle                        */
+    SPEC_OPT_HEAD_PAIR = 7       /* 1: levels of more than 128 nodes run the head GEMM on pairs of CTAs
+                                  (tcgen05.mma.cta_group::2: 256 node rows per tile, each CTA loads half
+                                  of the weight box); 0: one CTA per tile; -1 (default): pairs for
+                                  levels of at least 512 nodes whose padding to a multiple of 256 is at
+                                  most a tenth                                                  */
 };
 
 typedef struct spec_handle_s *spec_handle_t;

@@ -23,6 +23,7 @@ SPEC_BF16, SPEC_F32 = 0, 1
 SPEC_OPT_GEMM_IMPL, SPEC_OPT_HEAD_BLOCK_N, SPEC_OPT_PROJ_BLOCK_N, SPEC_OPT_PROFILE, SPEC_OPT_FP8_MAX_ROWS = 0, 1, 2, 3, 4
 SPEC_OPT_HEAD_SWAP_MAX_ROWS = 5
 SPEC_OPT_GEMM_PRODUCERS = 6
+SPEC_OPT_HEAD_PAIR = 7
 
 EXPORTS = [
     "spec_version", "spec_status_str", "spec_last_cuda_error", "spec_create", "spec_destroy", "spec_set_option",

@@ -10,7 +10,7 @@ _ROOT = os.path.dirname(_PKG)
 CSRC = os.path.join(_PKG, "csrc")
 INCLUDE = os.path.join(_ROOT, "include")
 LIB_PATH = os.path.join(_PKG, "libspec_b200.so")
-SOURCES = ["spec_api.cu", "verify_kernels.cu", "draft_kernels.cu", "fp8_kernels.cu", "gemm_tcgen05.cu", "gemm_simt.cu"]
+SOURCES = ["spec_api.cu", "verify_kernels.cu", "draft_kernels.cu", "fp8_kernels.cu", "gemm_tcgen05.cu", "gemm_pair.cu", "gemm_simt.cu"]
 
 
 def _newest_source_mtime() -> float:

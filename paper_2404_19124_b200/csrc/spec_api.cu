@@ -38,6 +38,7 @@ struct spec_handle_s {
     int profile;
     int fp8_max_rows;                      // SPEC_OPT_FP8_MAX_ROWS
     int swap_max_rows;                     // SPEC_OPT_HEAD_SWAP_MAX_ROWS
+    int head_pair;                         // SPEC_OPT_HEAD_PAIR
     const void *head8[SPEC_MAX_HEADS];     // e4m3 copies of the heads (caller-owned), null: none
     const float *head8_scale[SPEC_MAX_HEADS];
     int vp_rank, vp_ranks;                 // vocabulary-parallel heads: this handle's shard (vp_ranks 1: none)
@@ -64,6 +65,7 @@ struct DraftPlan {
     int proj_splits[SPEC_MAX_HEADS];   // > 0: swapped split-K projection (few parent rows); 0: plain
     bool use_fp8[SPEC_MAX_HEADS];      // the level's head runs on the e4m3 copy of its weights
     bool swapped[SPEC_MAX_HEADS];      // the level's head runs with the operands swapped (few nodes: weight stream)
+    bool paired[SPEC_MAX_HEADS];       // the level's head runs on CTA pairs (more than 128 nodes: tensor-bound)
     size_t seq_done;                   // byte offset of the per-sequence counters of the folded prune
     int header_words;                  // int32 words cleared at the start of a draft
     size_t xchg;                       // vocabulary-parallel heads: byte offset of the rank slots
@@ -87,8 +89,24 @@ bool head_swapped_for(const spec_handle_s *h, int rows) {
     return rows <= 8 || (rows <= 32 && h->head_rows >= 4 * 128 * num_sms());
 }
 
+// Levels of more than 128 nodes (several 128-row tiles per weight tile) may run on CTA pairs.
+// A pair's tile has 256 node rows, so a level whose row count is not a multiple of 256 pays for the padding:
+// 384 rows run as 512 (measured 100 against 88 us, V = 32000), 512 / 768 / 2048 / 6144 rows gain 4-9 %.
+// Automatic: at least 512 rows and at most a tenth of padding.
+bool head_paired_for(const spec_handle_s *h, int rows) {
+    if (h->gemm_impl != 0 || h->head_block_n != 0 || rows <= 128 || h->head_pair == 0) return false;
+    if (h->head_pair == 1) return true;
+    const int padded = (rows + 255) / 256 * 256;
+    return rows >= 512 && 10 * padded <= 11 * rows;
+}
+
 // Partial lists per row that the head of `rows` nodes leaves for the merge, and its tile width.
 int head_parts_for(const spec_handle_s *h, int rows, bool swapped, int *block_n_out) {
+    if (head_paired_for(h, rows)) {
+        const int bn = pair_block_n(rows, h->head_rows);
+        if (block_n_out) *block_n_out = bn;
+        return (h->head_rows + bn - 1) / bn;
+    }
     if (swapped) {
         if (block_n_out) *block_n_out = 128;
         return swapped_head_parts(rows, h->head_rows);
@@ -168,6 +186,7 @@ int make_draft_plan(const spec_handle_s *h, int B, const int32_t *topk, int K, D
                         w.d_inner <= 16384 && h->vp_ranks == 1;
         if (p->use_fp8[l] && p->N[l] > max_fp8_rows) max_fp8_rows = p->N[l];
         p->swapped[l] = !p->use_fp8[l] && head_swapped_for(h, p->N[l]);
+        p->paired[l] = !p->use_fp8[l] && !h->profile && head_paired_for(h, p->N[l]);
     }
     for (int l = 0; l < p->n; ++l) {
         y.state[l] = off;
@@ -228,6 +247,7 @@ int run_head_partials(const spec_handle_s *h, const void *states, const void *Wo
     e.part_idx = part_idx;
     e.part_ms = part_ms;
     e.topk = topk;
+    if (head_paired_for(h, rows)) return launch_head_pair(states, Wout, rows, w.V, w.d_inner, block_n, e, err, st);
     if (head_swapped_for(h, rows)) {
         e.mode = 3;
         return launch_gemm_tc(Wout, states, w.V, rows, w.d_inner, (rows + 15) / 16 * 16, e, err, st);
@@ -375,6 +395,7 @@ int spec_create(spec_handle_t *out, const spec_weights_t *w) {
     h->profile = 0;
     h->fp8_max_rows = 128;
     h->swap_max_rows = -1;
+    h->head_pair = -1;
     h->vp_rank = 0;
     h->vp_ranks = 1;
     h->vocab_offset = 0;
@@ -420,6 +441,10 @@ int spec_set_option(spec_handle_t h, int option, int value) {
         case SPEC_OPT_FP8_MAX_ROWS:
             if (value < 0 || value > (1 << 24)) return SPEC_ERR_INVALID_ARG;
             h->fp8_max_rows = value;
+            return SPEC_OK;
+        case SPEC_OPT_HEAD_PAIR:
+            if (value < -1 || value > 1) return SPEC_ERR_INVALID_ARG;
+            h->head_pair = value;
             return SPEC_OK;
         case SPEC_OPT_GEMM_PRODUCERS:
             if (value != 1 && value != 2) return SPEC_ERR_INVALID_ARG;
@@ -556,7 +581,16 @@ int spec_draft(spec_handle_t h, const void *ctx_state, const int32_t *last_tok, 
         // launch: its weight tiles follow the head's through the same ring and one kernel boundary less
         // lies on the critical path (with per-kernel profiling it stays a launch of its own).
         proj_done = false;
-        if (h->gemm_impl == 0 && !h->profile) {
+        if (p.paired[l]) {
+            // tensor-bound level: the head on CTA pairs; the next level's projection follows as a launch of its own
+            const GemmCall hc = make_head_call(h, p, ws, l, topk[l]);
+            rc = launch_head_pair(hc.A, hc.B, hc.M, hc.N, hc.Kd, hc.block_n, hc.epi, err, st);
+            if (rc == SPEC_OK && l + 1 < p.n) {
+                const GemmCall pc = proj_call(l + 1);
+                rc = launch_gemm_tc_jobs(&pc, 1, err, st);
+                proj_done = rc == SPEC_OK;
+            }
+        } else if (h->gemm_impl == 0 && !h->profile) {
             GemmCall c[2];
             c[0] = make_head_call(h, p, ws, l, topk[l]);
             const bool pair = l + 1 < p.n;

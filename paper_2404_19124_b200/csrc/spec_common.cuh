@@ -130,6 +130,11 @@ struct GemmCall {
 int launch_gemm_tc_jobs(const GemmCall *calls, int n_calls, int32_t *err, cudaStream_t st, int32_t *clear = nullptr,
                         int clear_words = 0);
 
+// ---- the tensor-bound head on CTA pairs (gemm_pair.cu) --------------------------------------------
+int pair_block_n(int rows, int vocab_rows);
+int launch_head_pair(const void *states, const void *W, int rows, int V, int Kd, int block_n, const GemmEpilogue &epi,
+                     int32_t *err, cudaStream_t st);
+
 // ---- debug CUDA-core GEMM (gemm_simt.cu) ------------------------------------------------
 int launch_gemm_simt(const void *A, const void *B, int M, int N, int Kd, float *C, int ldc, cudaStream_t st);
 // Builds the per-tile partial lists (same format as the fused epilogue) from full logits.

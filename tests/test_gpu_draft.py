@@ -81,17 +81,21 @@ def _check_topk_rows(tok, logp, logits, k):
 
 
 # impl 0: tensor cores, nodes as columns of the MMA for up to 128 rows (the weight-stream form); 1: CUDA-core
-# debug GEMM; 2: tensor cores with one thread per node row at every size
-@pytest.mark.parametrize("impl", [0, 1, 2])
+# debug GEMM; 2: tensor cores with one thread per node row at every size; 3: CTA pairs above 128 rows
+@pytest.mark.parametrize("impl", [0, 1, 2, 3])
 @pytest.mark.parametrize("rows,V,d,k", [(1, 1024, 256, 4), (12, 1024, 256, 2), (130, 1000, 128, 8),
                                         (40, 8000, 512, 6), (5, 64, 64, 8), (3, 40, 64, 1), (16, 32000, 256, 6),
-                                        (96, 20040, 192, 3), (128, 5000, 64, 5), (33, 1000, 200, 8), (64, 129, 72, 7)])
+                                        (96, 20040, 192, 3), (128, 5000, 64, 5), (33, 1000, 200, 8), (64, 129, 72, 7),
+                                        (384, 2048, 256, 3), (257, 1096, 64, 6), (700, 3000, 192, 2)])
 def test_head_topk_matches_oracle(B, impl, rows, V, d, k):
+    if impl == 3 and rows <= 128:
+        pytest.skip("pairs serve levels of more than 128 rows")
     cfg = small_cfg(d_base=d, d_inner=d, V=V, topk=(2, 2), seed=rows * 7 + k)
     sw, ow, gw = _setup(cfg)
     h = B.spec_create(gw)
-    B.spec_set_option(h, B.SPEC_OPT_GEMM_IMPL, impl & 1)
+    B.spec_set_option(h, B.SPEC_OPT_GEMM_IMPL, impl & 1 if impl < 3 else 0)
     B.spec_set_option(h, B.SPEC_OPT_HEAD_SWAP_MAX_ROWS, 0 if impl == 2 else 128)
+    B.spec_set_option(h, B.SPEC_OPT_HEAD_PAIR, 1 if impl == 3 else 0)
     S = _states(rows, d, 4)
     tok, logp, ws = B.spec_head_topk(h, 0, S.cuda(), k)
     assert B.spec_poll_error(ws) == 0
@@ -149,6 +153,7 @@ def _draft_and_check(B, cfg, seqs=None, impl=0, check_levels=False, tie_weights=
     B.spec_set_option(h, B.SPEC_OPT_GEMM_IMPL, impl)
     if swap is not None:   # levels of up to `swap` nodes run the head with the nodes as MMA columns (0: none)
         B.spec_set_option(h, B.SPEC_OPT_HEAD_SWAP_MAX_ROWS, swap)
+        B.spec_set_option(h, B.SPEC_OPT_HEAD_PAIR, 1 if swap else 0)   # and levels of > 128 nodes on CTA pairs / not
     if fp8:      # levels of up to 128 nodes multiply in e4m3 and re-score a short list exactly
         B.spec_attach_fp8_heads(h)
         if fp8_rows is not None:   # also levels with more than the default 128 nodes

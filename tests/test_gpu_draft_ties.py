@@ -48,6 +48,7 @@ def test_all_scores_equal_returns_the_lowest_leaves_in_order(B, topk, K, fp8):
         B.spec_set_option(h, B.SPEC_OPT_FP8_MAX_ROWS, 4096)
     else:   # the levels of up to 128 nodes in the form with the nodes as MMA columns
         B.spec_set_option(h, B.SPEC_OPT_HEAD_SWAP_MAX_ROWS, 128 if K % 2 else 0)
+        B.spec_set_option(h, B.SPEC_OPT_HEAD_PAIR, 1 if K % 2 else 0)      # and CTA pairs above 128 nodes
     ct, lp, ws = B.spec_draft(h, ctx.cuda(), tok.cuda(), cfg.topk, K)
     assert B.spec_poll_error(ws) == 0
     want = [_leaf_digits(i, topk) for i in range(K)]
@@ -81,6 +82,7 @@ def test_tie_across_the_K_boundary_keeps_the_lower_leaf(B, topk, K, Bn, V, d, fp
         B.spec_set_option(h, B.SPEC_OPT_FP8_MAX_ROWS, 4096)
     else:
         B.spec_set_option(h, B.SPEC_OPT_HEAD_SWAP_MAX_ROWS, 128 if Bn % 4 == 0 else 0)
+        B.spec_set_option(h, B.SPEC_OPT_HEAD_PAIR, 1 if Bn % 4 == 0 else 0)
     ct, lp, ws = B.spec_draft(h, ctx.cuda(), tok.cuda(), cfg.topk, K)
     assert B.spec_poll_error(ws) == 0
     ct, lp = ct.cpu().numpy(), lp.cpu().numpy()

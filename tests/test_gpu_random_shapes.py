@@ -46,6 +46,7 @@ def test_draft_random_shapes(B, case):
         B.spec_attach_fp8_heads(h)          # every third case through the e4m3 heads
     elif case % 3 == 1:
         B.spec_set_option(h, B.SPEC_OPT_HEAD_SWAP_MAX_ROWS, 128)   # every third case: nodes as MMA columns
+        B.spec_set_option(h, B.SPEC_OPT_HEAD_PAIR, 1)              # ... up to 128 nodes, CTA pairs above
     cand_tok, cand_logp, ws = B.spec_draft(h, ctx.cuda(), tok.cuda(), cfg.topk, cfg.K)
     assert B.spec_poll_error(ws) == 0
     ct, lp = cand_tok.cpu().numpy(), cand_logp.cpu().numpy()
