@@ -70,8 +70,7 @@ enum spec_option {
     SPEC_OPT_HEAD_PAIR = 7       /* 1: levels of more than 128 nodes run the head GEMM on pairs of CTAs
                                   (tcgen05.mma.cta_group::2: 256 node rows per tile, each CTA loads half
                                   of the weight box); 0: one CTA per tile; -1 (default): pairs for
-                                  levels of at least 512 nodes whose padding to a multiple of 256 is at
-                                  most a tenth                                                  */
+                                  levels whose padding to a multiple of 256 nodes is at most a tenth */
 };
 
 typedef struct spec_handle_s *spec_handle_t;

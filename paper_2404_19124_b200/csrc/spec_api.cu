@@ -91,13 +91,13 @@ bool head_swapped_for(const spec_handle_s *h, int rows) {
 
 // Levels of more than 128 nodes (several 128-row tiles per weight tile) may run on CTA pairs.
 // A pair's tile has 256 node rows, so a level whose row count is not a multiple of 256 pays for the padding:
-// 384 rows run as 512 (measured 100 against 88 us, V = 32000), 512 / 768 / 2048 / 6144 rows gain 4-9 %.
-// Automatic: at least 512 rows and at most a tenth of padding.
+// 384 rows run as 512 (measured 100 against 88 us, V = 32000), 256 / 512 / 768 / 2048 / 6144 rows gain 4-9 %.
+// Automatic: at most a tenth of padding (233-256 rows, 466-512, 699-768, ...).
 bool head_paired_for(const spec_handle_s *h, int rows) {
     if (h->gemm_impl != 0 || h->head_block_n != 0 || rows <= 128 || h->head_pair == 0) return false;
     if (h->head_pair == 1) return true;
     const int padded = (rows + 255) / 256 * 256;
-    return rows >= 512 && 10 * padded <= 11 * rows;
+    return 10 * padded <= 11 * rows;
 }
 
 // Partial lists per row that the head of `rows` nodes leaves for the merge, and its tile width.
