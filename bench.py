@@ -214,10 +214,62 @@ class Workload:
         self.draft(i)
         self.verify(i)
 
+    def capture(self):
+        """n_rot consecutive steps (one per logits buffer) recorded once as a CUDA graph.  Leaves `graph` None
+        when stream capture is not available; the steps are then launched call by call."""
+        torch, c = self.torch, self.cfg
+        self.graph = None
+        try:
+            cur = torch.cuda.current_stream()
+            gs = torch.cuda.Stream()
+            gs.wait_stream(cur)
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.stream(gs):
+                with torch.cuda.graph(g, stream=gs):
+                    for i in range(self.n_rot):
+                        self.B.spec_draft(self.h, self.ctx, self.tok, c.topk, c.K, cand_tok=self.cand, cand_logp=self.logp,
+                                          workspace=self.ws, stream=gs)
+                        self.B.spec_verify(self.cand, self.rot[i], accept_len=self.acc, best_cand=self.best,
+                                           next_tok=self.nxt, workspace=self.vws, stream=gs)
+            cur.wait_stream(gs)
+            self.graph = g
+        except RuntimeError as e:
+            sys.stderr.write(f"CUDA graph capture not available, steps are launched call by call: {e}\n")
+        return self.graph is not None
+
+    def run_steps(self, steps: int):
+        """Exactly `steps` steps on the current stream: whole replays of the captured graph, the rest call by call."""
+        g = getattr(self, "graph", None)
+        reps = steps // self.n_rot if g is not None else 0
+        for _ in range(reps):
+            g.replay()
+        for i in range(steps - reps * self.n_rot):
+            self.step(i)
+
+    def launch_form(self) -> str:
+        if getattr(self, "graph", None) is None:
+            return "call by call (spec_draft, spec_verify)"
+        return (f"CUDA graph of {self.n_rot} steps (spec_draft + spec_verify captured once, one logits buffer each) "
+                f"replayed; steps beyond a whole number of replays call by call")
+
     def close(self):
+        self.graph = None
         self.B.spec_destroy(self.h)
         self.rot = self.sw = self.ws = None
         self.torch.cuda.empty_cache()
+
+
+def time_steps(torch, W: "Workload", steps: int, warm: int = 5) -> float:
+    """Milliseconds per step of W.run_steps(steps), CUDA events on the current stream."""
+    stream = torch.cuda.current_stream()
+    W.run_steps(warm)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    W.run_steps(steps)
+    e1.record(stream)
+    torch.cuda.synchronize()
+    return e0.elapsed_time(e1) / steps
 
 
 def time_loop(torch, fn, iters: int, warm: int = 3) -> float:
@@ -273,7 +325,10 @@ def verify_roofline(W: "Workload", ms: float, ms_early: float, peaks, traffic=No
 def workload_entry(W: "Workload", peaks, iters: int, world: int, shard):
     """Step, draft and verify times of one workload and the roofline fractions of its dominant head and of verify."""
     torch, cfg = W.torch, W.cfg
-    step_ms = time_loop(torch, W.step, iters)
+    direct_ms = time_loop(torch, W.step, iters)
+    if getattr(W, "graph", None) is None:
+        W.capture()
+    step_ms = time_steps(torch, W, iters) if W.graph is not None else direct_ms
     draft_ms = time_loop(torch, W.draft, iters)
     verify_ms = time_loop(torch, W.verify, iters)
     early_ms = time_loop(torch, lambda i: W.verify(i, early=True), iters)
@@ -285,7 +340,9 @@ def workload_entry(W: "Workload", peaks, iters: int, world: int, shard):
         heads.append(head_roofline(cfg, cfg.nodes(l), ms, peaks))
     tau = float(W.acc.float().mean().item()) + 1.0
     return {"B": cfg.B, "K": cfg.K, "topk": list(cfg.topk), "V": cfg.V, "d_inner": cfg.d_inner, "steps_timed": iters,
-            "step_us": round(step_ms * 1e3, 2), "draft_us": round(draft_ms * 1e3, 2), "verify_us": round(verify_ms * 1e3, 2),
+            "step_us": round(step_ms * 1e3, 2), "step_launch": W.launch_form(),
+            "step_us_call_by_call": round(direct_ms * 1e3, 2),
+            "draft_us": round(draft_ms * 1e3, 2), "verify_us": round(verify_ms * 1e3, 2),
             "verify_early_exit_us": round(early_ms * 1e3, 2),
             "sequences_per_s": shard.whole_job_rate(cfg.B, world, step_ms * 1e-3),
             "dominant_head": heads[last], "heads": [{"rows": cfg.nodes(l), "bound": hd["bound"], "us": hd["us"],
@@ -436,8 +493,7 @@ def main():
         barrier()
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         e0.record(stream)
-        for i in range(steps):
-            step(i)
+        W.run_steps(steps)
         e1.record(stream)
         barrier()
         ms = max_over_ranks(e0.elapsed_time(e1) / steps)
@@ -446,6 +502,9 @@ def main():
     # ---------------------------------------------------------------- device-resident timing
     for i in range(args.warmup):
         step(i)
+    W.capture()                  # (after the warm-up: every tensor map and attribute the launches need exists)
+    launch_form = W.launch_form()
+    W.run_steps(n_rot)
     ms_step, clocks = timed_region(args.steps)
     assert B.spec_poll_error(ws) == 0
     tau = float(acc.float().mean().item()) + 1.0
@@ -503,34 +562,10 @@ def main():
     e2e_ms = max_over_ranks((time.perf_counter() - t0) * 1e3 / e2e_steps)
     del d_logits, h_rot
 
-    # ---------------------------------------------------------------- the same steps as one CUDA graph
-    # n_rot steps (one per logits buffer) captured once and replayed: what is left when the host's launch
-    # calls are taken out of the picture
-    graph_ms = None
-    try:
-        gs = torch.cuda.Stream()
-        gs.wait_stream(stream)
-        graph = torch.cuda.CUDAGraph()
-        with torch.cuda.stream(gs):
-            with torch.cuda.graph(graph, stream=gs):
-                for i in range(n_rot):
-                    B.spec_draft(h, ctx, tok, cfg.topk, K, cand_tok=cand, cand_logp=logp, workspace=ws, stream=gs)
-                    B.spec_verify(cand, rot[i], accept_len=acc, best_cand=best, next_tok=nxt, workspace=vws, stream=gs)
-            replays = max(3, min(args.steps, 400) // n_rot)
-            for _ in range(3):
-                graph.replay()
-            gs.synchronize()
-            g0, g1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            g0.record(gs)
-            for _ in range(replays):
-                graph.replay()
-            g1.record(gs)
-            gs.synchronize()
-        graph_ms = max_over_ranks(g0.elapsed_time(g1) / (replays * n_rot))
-        stream.wait_stream(gs)
-        del graph
-    except RuntimeError as e:      # capture not available: the key stays null, nothing else depends on it
-        sys.stderr.write(f"graph replay skipped: {e}\n")
+    # ---------------------------------------------------------------- the same steps launched call by call
+    # (the timed region above replays a CUDA graph when capture is available)
+    direct_steps = max(3, min(args.steps, 200))
+    direct_ms = max_over_ranks(time_loop(torch, step, direct_steps))
     assert B.spec_poll_error(ws) == 0
 
     # ---------------------------------------------------------------- host time of one spec_draft call
@@ -710,8 +745,9 @@ def main():
                             "frac_of_burst": round(2.0 * bk_rows * cfg.d_inner * V / (bk_ms * 1e-3) / 1e12 / peaks["bf16_tflops"], 3)},
         "step_with_e4m3_heads": {"ms_per_step": round(fp8_step_ms, 5), "value": shard.whole_job_rate(Bn, world, fp8_step_ms * 1e-3),
                                  "what": "optional mode: e4m3 head copies on the weight-bound levels, short list re-scored in bf16"},
-        "graph_replay": {"ms_per_step": None if graph_ms is None else round(graph_ms, 5),
-                         "what": "the same draft + verify steps captured in one CUDA graph and replayed"},
+        "launch": launch_form,
+        "call_by_call": {"ms_per_step": round(direct_ms, 5), "steps": direct_steps,
+                         "what": "the same steps as separate spec_draft / spec_verify calls on the stream, no graph"},
         "kernel_us": kernels, "kernel_us_note": "separate-kernel form bracketed by events (adds 2-3 us per kernel and takes "
                                                 "away the overlap of consecutive kernels); the timed step launches the next "
                                                 "level's projection with the head",
