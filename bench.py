@@ -656,7 +656,7 @@ def main():
 
     # ---------------------------------------------------------------- vocabulary-parallel heads (N > 1 only)
     # The optional mode for small batches: every rank holds 1/N of each head's vocabulary rows, the per-level
-    # lists are all-gathered with NCCL (no multicast loads anywhere), every rank ends with the same candidates.
+    # lists are all-gathered with NCCL, every rank ends with the same candidates.
     # Whole-draft time with the exchange inside, max over ranks; never part of `value`.
     vocab_parallel = None
     if dist is not None:

@@ -261,7 +261,7 @@ int spec_verify_static(const int32_t *cand_tok, const void *base_logits, int log
  *                            A collective enqueued on the draft's stream (NCCL all-gather) orders this by
  *                            itself; with direct peer stores the writer must first learn (an event, a flag, a
  *                            barrier per level) that the peer's merge of the previous level is done.  Peer
- *                            traffic is plain loads / stores or NCCL; the library issues no multicast loads.
+ *                            traffic is plain loads / stores or NCCL; every TMA copy the library issues has one destination CTA.
  *   spec_draft_vp_local / _merge  arguments as spec_draft; the same B, topk, K and workspace for every
  *                            step of one draft (workspace size: spec_draft_workspace_bytes on the sharded
  *                            handle).  cand_tok / cand_logp are written by the merge of the last level

@@ -10,11 +10,11 @@
 //
 // Roles per CTA (224 threads) as in gemm_tc_kernel: warps 0 and 6 issue the TMA copies of this CTA's operand
 // halves (their completion bytes go to the barrier of the pair's first CTA), warp 1 of the first CTA issues the
-// MMAs for both and releases ring slots and accumulators in both CTAs with multicast commits, warps 2-5 of
+// MMAs for both and releases ring slots and accumulators in both CTAs with commits that arrive in both, warps 2-5 of
 // either CTA run the fused top-k / log-sum-exp epilogue on their own 128 rows of the accumulator (tc_gemm.cuh,
 // one thread per node row) and then tell the first CTA that the accumulator slot is free.  Every wait on an
 // mbarrier is bounded; every thread of both CTAs reaches the cluster barrier at the end whatever happened, TMEM is
-// freed behind it.  No TMA load here is a multicast load.
+// freed behind it.  Every TMA copy here has one destination: the shared memory of the CTA that issued it.
 #include <cuda.h>
 
 #include <mutex>
@@ -94,7 +94,7 @@ __device__ __forceinline__ void abort_grace() {
 }
 
 // This CTA's box of a pair's tile; the completion bytes are counted on `bar_cluster_addr` (a barrier of the pair's
-// first CTA).  Not a multicast load: every CTA fetches its own box into its own shared memory.
+// first CTA).  Every CTA fetches its own box into its own shared memory; nothing is broadcast across the pair.
 __device__ __forceinline__ void tma_load_2d_pair(void *dst, const CUtensorMap *map, int c0, int c1, uint32_t bar_cluster_addr) {
     asm volatile(
         "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
