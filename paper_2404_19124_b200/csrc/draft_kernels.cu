@@ -24,6 +24,18 @@ __global__ void __launch_bounds__(kRowThreads, 2) mix_ln_gelu_kernel(MixArgs m) 
     else mix_ln_gelu_row<kRowThreads, 2, 2, BlockSync>(m, blockIdx.x, threadIdx.x, red);
 }
 
+// Rows of 2049 to 4096 elements in levels of at most one CTA per SM: 512 threads, one 8-element group each.  The
+// step is a chain of dependent latencies (loads, two reductions, sixteen erf evaluations per thread with 256
+// threads), so halving the per-thread work shortens it: 13B-shaped draft 3-5 us faster than with 256 threads.  At
+// most 72 registers, so that the CTA fits beside a resident GEMM CTA.
+constexpr int kWideRowThreads = 512;
+__global__ void __maxnreg__(72) mix_ln_gelu_512_kernel(MixArgs m) {
+    __shared__ float red[32];
+    griddep_launch();
+    griddep_wait();
+    mix_ln_gelu_row<kWideRowThreads, 1, 1, BlockSync>(m, blockIdx.x, threadIdx.x, red);
+}
+
 // The same for levels with more nodes than one wave of the kernel above holds: one 8-element group in
 // flight per thread and at most 80 registers, so three CTAs share an SM and the level stays one wave.
 __global__ void __launch_bounds__(kRowThreads, 3) mix_ln_gelu_many_kernel(MixArgs m) {
@@ -121,6 +133,19 @@ __global__ void __launch_bounds__(kRowThreads, 2) merge_mix_kernel(MergeMixArgs 
         mix_children<kRowThreads, 2, kFusedBatch, BlockSync>(a.mix, r, r * a.merge.topk, a.merge.topk, sc.out_id, red_a, red_b, tid);
 }
 
+// Rows of 2049 to 4096 elements: 512 threads, one 8-element group each, like mix_ln_gelu_512_kernel (single-
+// candidate chain at the 13B widths 210 -> 203 us per draft, at the 34B widths 278 -> 269 us).  72 registers at
+// most, so that the CTA fits beside a resident GEMM CTA.
+__global__ void __maxnreg__(72) merge_mix_512_kernel(MergeMixArgs a) {
+    __shared__ Scratch sc;
+    __shared__ float red_a[kWideRowThreads / 32 * kFusedBatch], red_b[kWideRowThreads / 32 * kFusedBatch];
+    griddep_launch();
+    griddep_wait();
+    const int r = blockIdx.x, tid = threadIdx.x;
+    merge_expand_row<kWideRowThreads, BlockSync>(a.merge, r, tid, &sc);
+    mix_children<kWideRowThreads, 1, kFusedBatch, BlockSync>(a.mix, r, r * a.merge.topk, a.merge.topk, sc.out_id, red_a, red_b, tid);
+}
+
 // Vocabulary-parallel head: one warp per row folds the n_ranks raw lists (see launch_merge_shards).
 // Lane i owns entries i and i + 32 of the row's n_ranks * topk <= 64 candidates.
 constexpr int kShardRowsPerCta = 4;
@@ -195,6 +220,8 @@ int launch_mix_ln_gelu(const MixArgs &m, int rows, cudaStream_t st) {
     const int d_inner = m.d;
     if (d_inner <= 8 * kRowThreads * 2 && rows > num_sms()) {
         SPEC_CUDA_TRY(launch_pdl(mix_ln_gelu_many_kernel, dim3(rows), dim3(kRowThreads), 0, st, m));
+    } else if (d_inner <= 8 * kWideRowThreads && d_inner > 8 * kRowThreads) {
+        SPEC_CUDA_TRY(launch_pdl(mix_ln_gelu_512_kernel, dim3(rows), dim3(kWideRowThreads), 0, st, m));
     } else if (d_inner <= 8 * kRowThreads * 2) {
         SPEC_CUDA_TRY(launch_pdl(mix_ln_gelu_kernel, dim3(rows), dim3(kRowThreads), 0, st, m));
     } else if (d_inner <= 8 * kRowThreads * 8) {
@@ -226,6 +253,10 @@ int launch_merge_mix(const MergeArgs &g, const MixArgs &m, int rows, cudaStream_
     if (m.d > 8 * kRowThreads * 2 || m.S8_out != nullptr || g.lse_out != nullptr || g.seq_done != nullptr)
         return SPEC_ERR_SHAPE;
     MergeMixArgs a{g, m};
+    if (m.d > 8 * kRowThreads && m.d <= 8 * kWideRowThreads) {
+        SPEC_CUDA_TRY(launch_pdl(merge_mix_512_kernel, dim3(rows), dim3(kWideRowThreads), 0, st, a));
+        return SPEC_OK;
+    }
     SPEC_CUDA_TRY(launch_pdl(merge_mix_kernel, dim3(rows), dim3(kRowThreads), 0, st, a));
     return SPEC_OK;
 }

@@ -183,6 +183,17 @@ verify_accept_kernel(const int32_t *cand_tok, const float *pval, const int32_t *
         key_s = 0u;
         if (b == 0 && err != nullptr) *err = 0;
     }
+    // The step is a handful of dependent round trips to L2, so every load that does not depend on another is
+    // requested before the first one is used: the tokens of this thread's first candidate now, a row's partials
+    // (values and indices alike) eight slots at a time.
+    constexpr int kBatch = 8;
+    int32_t ctok[SPEC_MAX_HEADS];
+    {
+        const int k0 = threadIdx.x;
+#pragma unroll
+        for (int j = 0; j < SPEC_MAX_HEADS; ++j)
+            ctok[j] = (k0 < K && j < n) ? __ldcg(cand_tok + ((size_t)b * K + k0) * n + j) : -1;
+    }
     for (int r = threadIdx.x; r < rows_b; r += blockDim.x) {
         const size_t gr = (size_t)b * rows_b + r;
         const size_t u0 = gr * slots;
@@ -192,11 +203,20 @@ verify_accept_kernel(const int32_t *cand_tok, const float *pval, const int32_t *
             chunks = (int)(((long long)(gr + 1) * vpr - 1) / vec_per_warp - ((long long)gr * vpr) / vec_per_warp) + 1;
         float best = -INFINITY;
         int arg = 0;   // a row without any value above -inf (all NaN) yields 0
-        for (int c = 0; c < chunks; ++c) {
-            const float v = __ldcg(pval + u0 + c);
-            if (v > best) {   // chunks ascend, so the first maximum wins
-                best = v;
-                arg = __ldcg(pidx + u0 + c);
+        for (int c0 = 0; c0 < chunks; c0 += kBatch) {
+            float v[kBatch];
+            int id[kBatch];
+#pragma unroll
+            for (int j = 0; j < kBatch; ++j) {
+                const bool in = c0 + j < chunks;
+                v[j] = in ? __ldcg(pval + u0 + c0 + j) : -INFINITY;
+                id[j] = in ? __ldcg(pidx + u0 + c0 + j) : 0;
+            }
+#pragma unroll
+            for (int j = 0; j < kBatch; ++j) {
+                const bool take = v[j] > best;   // chunks ascend, so the first maximum wins
+                best = take ? v[j] : best;
+                arg = take ? id[j] : arg;
             }
         }
         if (g_in_smem) g_s[r] = arg;
@@ -205,10 +225,23 @@ verify_accept_kernel(const int32_t *cand_tok, const float *pval, const int32_t *
     __syncthreads();
     const int32_t *gtab = g_in_smem ? g_s : g_out + (size_t)b * rows_b;
     for (int k = threadIdx.x; k < K; k += blockDim.x) {
-        const int32_t *c = cand_tok + ((size_t)b * K + k) * n;
         const int32_t *gk = gtab + k * (n + 1);
+        if (k != (int)threadIdx.x) {   // more candidates than threads: the later ones are fetched here
+#pragma unroll
+            for (int j = 0; j < SPEC_MAX_HEADS; ++j)
+                ctok[j] = j < n ? __ldcg(cand_tok + ((size_t)b * K + k) * n + j) : -1;
+        }
         int m = 0;
-        while (m < n && __ldcg(c + m) == gk[m]) ++m;
+        bool open = true;
+#pragma unroll
+        for (int j = 0; j < SPEC_MAX_HEADS; ++j) {
+            open = open && j < n && ctok[j] == gk[j];
+            m += open ? 1 : 0;
+        }
+        if (open && n > SPEC_MAX_HEADS) {   // longer candidates than the registers hold: one token at a time
+            const int32_t *c = cand_tok + ((size_t)b * K + k) * n;
+            while (m < n && __ldcg(c + m) == gk[m]) ++m;
+        }
         // longest prefix first, then the lowest candidate index
         atomicMax(&key_s, ((unsigned)m << 16) | (unsigned)(0xffff - k));
     }

@@ -58,7 +58,7 @@ def _run_and_compare(B, cand: torch.Tensor, logits: torch.Tensor, forms=(False, 
 
 @pytest.mark.parametrize("dtype", [torch.bfloat16, torch.float32])
 @pytest.mark.parametrize("shape", [(1, 8, 3, 1024), (3, 5, 2, 1000), (2, 3, 4, 1021), (2, 7, 1, 8), (1, 1, 1, 1),
-                                   (4, 2, 7, 4100), (2, 64, 4, 50264)])
+                                   (4, 2, 7, 4100), (2, 64, 4, 50264), (2, 20, 12, 96), (1, 300, 9, 64)])
 def test_verify_small_shapes(B, dtype, shape):
     Bn, K, n, V = shape
     g = torch.Generator().manual_seed(sum(shape))
