@@ -225,7 +225,9 @@ class Workload:
             gs.wait_stream(cur)
             g = torch.cuda.CUDAGraph()
             with torch.cuda.stream(gs):
-                with torch.cuda.graph(g, stream=gs):
+                # (thread-local capture mode: CUDA calls of other threads, e.g. a process group's watchdog, are
+                # none of this capture's business)
+                with torch.cuda.graph(g, stream=gs, capture_error_mode="thread_local"):
                     for i in range(self.n_rot):
                         self.B.spec_draft(self.h, self.ctx, self.tok, c.topk, c.K, cand_tok=self.cand, cand_logp=self.logp,
                                           workspace=self.ws, stream=gs)
