@@ -580,6 +580,12 @@ def main():
         e2e_step(i)
     torch.cuda.synchronize()
     e2e_ms = max_over_ranks((time.perf_counter() - t0) * 1e3 / e2e_steps)
+    # the grouped form must give what one call over the whole batch gives on the same logits
+    e2e_out = [t.clone() for t in h_out]
+    W.verify((e2e_steps - 1) % 2)
+    torch.cuda.synchronize()
+    for got, want in zip(e2e_out, (acc, best, nxt)):
+        assert torch.equal(got, want.cpu()), "end-to-end step: grouped verify differs from the whole-batch call"
     del d_logits, h_rot
 
     # ---------------------------------------------------------------- the same steps launched call by call
