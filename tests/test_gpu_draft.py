@@ -218,6 +218,17 @@ def test_draft_odd_shapes(B, topk, K, Bn, V, d_base, d, swap):
     assert chk.tolerated <= max(1, Bn // 5)
 
 
+@pytest.mark.parametrize("d", [2040, 2056, 4088, 4104])
+@pytest.mark.parametrize("topk,K", [((3, 2), 5), ((2, 1, 1), 2)])
+def test_draft_row_widths_round_the_thread_counts(B, topk, K, d):
+    """State rows just below and above 2048 and 4096 elements: the row steps change their thread count and the
+    number of element groups per thread there (256 threads, 512 threads, the wider kernels), in the separate mix
+    kernel (three children per node) and in the fused merge + mix kernel (one or two children per node)."""
+    cfg = small_cfg(d_base=72, d_inner=d, V=1000, topk=topk, K=K, B=3, seed=d % 97 + len(topk))
+    chk = _draft_and_check(B, cfg, check_levels=True)
+    assert chk.tolerated <= 1
+
+
 @pytest.mark.parametrize("topk,K", [((3, 2, 2, 1, 1), 9), ((2, 2, 2, 1, 1, 1, 1), 8), ((2, 1, 2, 1, 2, 1, 2, 1), 16)])
 def test_draft_code_model_head_counts(B, topk, K):
     """5, 7 (the code models of Sec. 4.3 / 4.4) and the maximum of 8 heads."""
